@@ -482,3 +482,116 @@ def test_explore_closed_forms():
     out = O.explore(np.tanh(rng.standard_normal((50, 4))).astype(np.float32), rng.uniform(0, 0.2, 50).astype(np.float32),
                     rng.standard_normal((50, 4)).astype(np.float32) * 10)
     assert out.min() >= -1.0 and out.max() <= 1.0
+
+
+# ---- input quantizer: the tie rule (round half to even, Eq. 1 on activations) ------------------
+
+def test_input_quantization_ties_go_to_even():
+    """delta = 2^-7 exactly, so x = (k + 1/2) * delta is an exact tie in binary32: the code is the even
+    neighbour (round-half-away would give +-1, +-2, +-3)."""
+    s, z = O.affine_params(-1.0, 0.9921875)
+    assert float(s) == 2.0 ** -7 and z == 0
+    d = 2.0 ** -7
+    x = np.array([0.5 * d, -0.5 * d, 1.5 * d, -1.5 * d, 2.5 * d, -2.5 * d, 3.5 * d, -3.5 * d, 126.5 * d, -127.5 * d],
+                 dtype=np.float32)
+    assert O.quantize_input_f32(x, s, z).tolist() == [0, 0, 2, -2, 2, -2, 4, -4, 126, -128]
+    # with a zero-point: the tie is decided before the offset is added (code = rne(x/delta) + z)
+    s2, z2 = O.affine_params(0.0, 255 * d)
+    assert float(s2) == d and z2 == -128
+    x2 = np.array([0.5 * d, 1.5 * d, 2.5 * d, 254.5 * d], dtype=np.float32)
+    assert O.quantize_input_f32(x2, s2, z2).tolist() == [-128, -126, -126, 126]
+
+
+# ---- a convolutional policy through the whole sequencing code --------------------------------
+
+class _C:
+    def __init__(self, w, b, stride, in_hw):
+        self.kind, self.weight, self.bias, self.stride, self.in_hw = "conv", w, b, stride, in_hw
+
+
+def _conv_f64_im2col(x, w, b, stride):
+    """float64 convolution by explicit patch extraction + matmul (independent of the C loops)."""
+    B, Cc, H, W = x.shape
+    Oc, _, KH, KW = w.shape
+    OH, OW = (H - KH) // stride + 1, (W - KW) // stride + 1
+    cols = np.empty((B, OH, OW, Cc * KH * KW), dtype=np.float64)
+    for oh in range(OH):
+        for ow in range(OW):
+            cols[:, oh, ow, :] = x[:, :, oh * stride:oh * stride + KH, ow * stride:ow * stride + KW].reshape(B, -1)
+    y = cols @ w.astype(np.float64).reshape(Oc, -1).T + (0 if b is None else b.astype(np.float64))
+    return y.transpose(0, 3, 1, 2)
+
+
+@pytest.mark.parametrize("stride,per_channel", [(1, False), (2, False), (1, True)])
+def test_tiny_conv_policy_end_to_end(stride, per_channel):
+    """uint8 frames 2x6x6 -> conv 3@3x3 -> FC 4 -> 2 Q-values through quantize_policy / forward.
+    Holds: the u8 activation parameters, the conv accumulators against im2col + numpy int64, the
+    (c, h, w) flatten into the first FC against an explicit index loop, the f64 conv against an
+    im2col product, and the int8 outputs against the un-quantized network within the propagated bound."""
+    rng = np.random.default_rng(50 + stride)
+    Cc, H, W, Oc, KH = 2, 6, 6, 3, 3
+    OH = (H - KH) // stride + 1
+    w0 = (rng.standard_normal((Oc, Cc, KH, KH)) * (2.0 / (Cc * KH * KH)) ** 0.5).astype(np.float32)
+    b0 = (rng.standard_normal(Oc) * 0.05).astype(np.float32)
+    feat = Oc * OH * OH
+    w1 = (rng.standard_normal((4, feat)) * (2.0 / feat) ** 0.5).astype(np.float32)
+    b1 = (rng.standard_normal(4) * 0.05).astype(np.float32)
+    w2 = (rng.standard_normal((2, 4)) * 0.7).astype(np.float32)
+    layers = [_C(w0, b0, stride, (H, W)), _L(w1, b1), _L(w2, None)]
+    if per_channel:
+        layers[0].per_channel = True
+    obs = rng.integers(0, 256, (40, Cc, H, W), dtype=np.uint8)
+    obs[0] = 0
+    obs[1] = 255
+
+    # un-quantized network: the C conv loop against an im2col matmul, then the rest by numpy
+    y_fp, inputs = O.forward_f64(layers, obs, "argmax", "u8")
+    x0 = obs.astype(np.float64) / 255.0
+    c_ref = np.maximum(_conv_f64_im2col(x0, w0, b0, stride), 0)
+    assert np.allclose(inputs[1].reshape(c_ref.shape), c_ref, rtol=1e-13, atol=1e-13)
+    h_ref = np.maximum(c_ref.reshape(40, -1) @ w1.astype(np.float64).T + b1, 0)
+    assert np.allclose(y_fp, h_ref @ w2.astype(np.float64).T, rtol=1e-12, atol=1e-12)
+
+    ranges = [(0.0, 1.0)] + [(float(v.min()), float(v.max())) for v in inputs[1:]]
+    qp = O.quantize_policy(layers, ranges, "argmax", "u8")
+    l0, l1 = qp.layers[0], qp.layers[1]
+    assert float(l0.s_a) == float(np.float32(1.0) / np.float32(255.0)) and l0.z_a == -128      # u8 frames mean u/255
+    y_q, act, trace = O.forward(qp, obs)
+
+    # conv accumulators: im2col + int64 matmul on (u - 128) - z_a = u
+    cols = _im2col(obs.astype(np.int64), KH, KH, stride)
+    zw = np.asarray(l0.z_w, dtype=np.int64).reshape(-1, 1) if per_channel else int(l0.z_w)
+    ref0 = cols @ (l0.w_q.astype(np.int64).reshape(Oc, -1) - zw).T + l0.bias_q
+    assert np.array_equal(trace[0][0], ref0.transpose(0, 3, 1, 2))
+    # flatten order into the FC: feature index = (c * OH + h) * OW + w
+    a1 = trace[0][1]
+    assert a1.shape == (40, Oc, OH, OH)
+    acc1 = np.zeros((40, 4), dtype=np.int64)
+    for c in range(Oc):
+        for h in range(OH):
+            for w_ in range(OH):
+                k = (c * OH + h) * OH + w_
+                acc1 += np.outer(a1[:, c, h, w_].astype(np.int64) - l1.z_a, l1.w_q[:, k].astype(np.int64) - int(l1.z_w))
+    assert np.array_equal(trace[1][0], acc1 + l1.bias_q)
+    assert np.array_equal(act, np.argmax(y_q, axis=1))
+
+    # propagated quantization bound, layer by layer (frames are exact: eps_0 = 0)
+    for r in range(40):
+        a = x0[r].reshape(1, Cc, H, W)
+        eps = np.zeros_like(a)
+        sw0 = (np.asarray(l0.s_w, dtype=np.float64).reshape(-1, 1, 1) if per_channel else float(l0.s_w))
+        P0 = (np.asarray(l0.P, dtype=np.float64).reshape(-1, 1, 1) if per_channel else float(l0.P))
+        ones = np.ones((Oc, Cc, KH, KH), dtype=np.float32)
+        e = (_conv_f64_im2col(eps, np.abs(w0), None, stride)[0]
+             + _conv_f64_im2col(np.abs(a) + eps, ones, None, stride)[0] * sw0 / 2 + P0 / 2)
+        a = c_ref[r].reshape(-1)
+        eps = e.reshape(-1) + float(l1.s_a) / 2
+        for i, (l, ql) in enumerate(zip(layers[1:], qp.layers[1:])):
+            Wm = l.weight.astype(np.float64)
+            e = np.abs(Wm) @ eps + (np.abs(a) + eps).sum() * float(ql.s_w) / 2 + float(ql.P) / 2
+            pre = Wm @ a + (0 if l.bias is None else l.bias.astype(np.float64))
+            if i == 0:
+                a = np.maximum(pre, 0)
+                eps = e + float(qp.layers[2].s_a) / 2
+        assert np.all(np.abs(y_q[r].astype(np.float64) - y_fp[r]) <= e * (1 + 1e-6) + 1e-6), (r, y_q[r], y_fp[r], e)
+    assert np.abs(y_q - y_fp).max() > 0
