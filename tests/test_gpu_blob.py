@@ -7,8 +7,21 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
+from oracle import oracle as O                      # noqa: E402
 from paper_1910_01055_b200 import binding as B      # noqa: E402
 from paper_1910_01055_b200 import workloads as W    # noqa: E402
+
+
+def _matches_checker(spec, obs_np, out, actions):
+    """the importing policy against the CPU checker run on the SENDER's fp32 weights"""
+    qp = O.quantize_policy(spec.layers, spec.input_ranges, spec.head, spec.obs_dtype)
+    y_ref, act_ref, _ = O.forward(qp, obs_np)
+    y = out.cpu().numpy()
+    assert np.all(np.abs(y - y_ref) <= 1e-5 * np.abs(y_ref) + 1e-30), float(np.abs(y - y_ref).max())
+    if spec.head != "tanh":
+        assert np.array_equal(y, y_ref)
+    if act_ref is not None:
+        assert np.array_equal(actions.cpu().numpy(), act_ref)
 
 
 def _policy(spec):
@@ -32,7 +45,8 @@ def test_blob_round_trip(kind):
     src_spec, dst_spec = _specs(kind, 3), _specs(kind, 4)
     dst_spec.input_ranges = src_spec.input_ranges            # activation ranges are part of the architecture's calibration
     src, dst = _policy(src_spec), _policy(dst_spec)
-    obs = torch.from_numpy(W.make_obs(src_spec, 300, seed=5)).cuda()
+    obs_np = W.make_obs(src_spec, 300, seed=5)
+    obs = torch.from_numpy(obs_np).cuda()
     want, want_act = src.forward(obs)
     other, _ = dst.forward(obs)
     assert not torch.equal(want, other)                      # different weights before the import
@@ -53,6 +67,7 @@ def test_blob_round_trip(kind):
     assert torch.equal(got, want)
     if want_act is not None:
         assert torch.equal(got_act, want_act)
+    _matches_checker(src_spec, obs_np, got, got_act)
     for i, l in enumerate(src_spec.layers):                   # codes, delta and zero-point arrived too
         a = torch.empty(l.weight.shape, dtype=torch.int8, device="cuda")
         b = torch.empty_like(a)
@@ -96,7 +111,8 @@ def test_blob_round_trip_per_channel_policy():
     src_spec, dst_spec = spec(3), spec(4)
     dst_spec.input_ranges = src_spec.input_ranges
     src, dst = _policy(src_spec), _policy(dst_spec)
-    obs = torch.from_numpy(W.make_obs(src_spec, 100, seed=5)).cuda()
+    obs_np = W.make_obs(src_spec, 100, seed=5)
+    obs = torch.from_numpy(obs_np).cuda()
     want, want_act = src.forward(obs)
     n = B.actorq_policy_blob_bytes(src.handle)
     blob = torch.empty(n, dtype=torch.uint8, device="cuda")
@@ -105,6 +121,7 @@ def test_blob_round_trip_per_channel_policy():
     got, got_act = dst.forward(obs)
     torch.cuda.synchronize()
     assert dst.status() == B.OK and torch.equal(got, want) and torch.equal(got_act, want_act)
+    _matches_checker(src_spec, obs_np, got, got_act)
     for i, l in enumerate(src_spec.layers):
         a = torch.empty(l.weight.shape, dtype=torch.int8, device="cuda")
         b = torch.empty_like(a)

@@ -1,9 +1,10 @@
 """actorq_policy_forward_host: chunked, pipelined forward on host buffers, held bit for bit against
-actorq_policy_forward on device buffers (which the parity tests hold against the CPU checker)."""
+actorq_policy_forward on device buffers and, on sampled rows, against the CPU checker."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as O
 from paper_1910_01055_b200 import binding as B
 from paper_1910_01055_b200 import workloads as W
 
@@ -19,6 +20,19 @@ def _built():
 
 def _policy(spec):
     return B.QuantizedPolicy(spec.head, spec.obs_dtype).quantize(B.layers_to_device(spec), spec.input_ranges)
+
+
+def _matches_checker(spec, obs_np, out_host, actions_host=None, max_rows=400):
+    """rows spread over every chunk of the call (first, last, and evenly spaced) against the checker"""
+    n = obs_np.shape[0]
+    idx = np.unique(np.concatenate([np.arange(min(n, 3)), np.arange(max(0, n - 3), n),
+                                    np.linspace(0, n - 1, min(n, max_rows)).astype(np.int64)]))
+    qp = O.quantize_policy(spec.layers, spec.input_ranges, spec.head, spec.obs_dtype)
+    y_ref, act_ref, _ = O.forward(qp, obs_np[idx])
+    y = out_host.numpy()[idx]
+    assert np.all(np.abs(y - y_ref) <= 1e-5 * np.abs(y_ref) + 1e-30), float(np.abs(y - y_ref).max())
+    if act_ref is not None:
+        assert np.array_equal(y, y_ref) and np.array_equal(actions_host.numpy()[idx], act_ref)
 
 
 @pytest.mark.parametrize("pinned", [True, False])
@@ -38,6 +52,7 @@ def test_host_forward_matches_device_forward_mlp(Bsz, pinned):
         torch.cuda.synchronize()
         assert pol.status() == B.OK
         assert torch.equal(out, ref.cpu())
+    _matches_checker(spec, obs.numpy(), out)
     pol.close()
 
 
@@ -57,6 +72,7 @@ def test_host_forward_conv_policy_with_actions_and_requantize_between():
         torch.cuda.synchronize()
         assert pol.status() == B.OK
         assert torch.equal(out, ref.cpu()) and torch.equal(act, ref_act.cpu())
+    _matches_checker(spec, obs.numpy(), out, act, max_rows=12)
     pol.close()
 
 

@@ -564,3 +564,49 @@ def test_forward_orders_after_the_kernel_that_produces_its_input(kind):
         assert pol.status() == B.OK
         assert torch.equal(out_a, ref_a) and torch.equal(out_b, ref_b)
     pol.close()
+
+
+def _edge_and_random_rows(Bsz, n_random, seed):
+    rng = np.random.default_rng(seed)
+    return np.unique(np.concatenate([np.arange(0, 130), np.arange(Bsz - 130, Bsz), rng.integers(0, Bsz, n_random)]))
+
+
+@pytest.mark.parametrize("per_channel", [False, True])
+@pytest.mark.parametrize("Bsz", [8192, 65536])
+def test_layer_pair_kernel_many_items_per_cta_pair(per_channel, Bsz):
+    """The paper's 2048-wide actor shape at batch sizes where every CTA pair of the layer kernel works
+    through many (tile pair, chunk) items in a row -- 3.5 per pair at 8192 rows, 28 at 65536 -- so the
+    alternating accumulators, the ring's phase wrap across items and the one-item-ahead prefetch of
+    row sums and column constants all run: sampled rows (first and last 130 plus random ones)
+    against the checker, every layer's accumulators and codes at 8192 rows."""
+    dims = [67, 2048, 2048, 21] if per_channel else [67, 2048, 2048, 2048, 21]
+    spec = W.mlp_policy("steady", dims, seed=73, head="tanh", nonzero_bias=True)
+    if per_channel:
+        for l in spec.layers:
+            l.weight *= np.linspace(0.2, 2.0, l.weight.shape[0], dtype=np.float32).reshape(-1, 1)
+            l.per_channel = True
+    W.calibrate(spec, 64, seed=73)
+    pol, qp, _ = _quantize_both(spec)
+    obs = W.make_obs(spec, Bsz, seed=73)
+    out, _ = _check_forward(pol, qp, spec, obs, _edge_and_random_rows(Bsz, 256, 73), check_layers=(Bsz == 8192))
+    again, _ = pol.forward(torch.from_numpy(obs).cuda())        # buffers and row-sum counters reused
+    torch.cuda.synchronize()
+    assert pol.status() == B.OK and torch.equal(out, again)
+    pol.close()
+
+
+@pytest.mark.parametrize("config,Bsz", [("mlp_wide", 65536), ("d4pg_humanoid", 40000)])
+def test_single_cta_fused_kernel_many_tiles_per_cta(config, Bsz):
+    """The single-CTA fused kernel with several tiles per CTA (512 and 313 tiles on 148 CTAs): its
+    persistent tile loop, the double-buffered first operand and the per-tile row sums, sampled rows
+    against the checker, and the whole batch bit for bit against the CTA-pair kernel."""
+    spec = W.build_config(config)
+    pol, qp, _ = _quantize_both(spec)
+    B.actorq_policy_set_fused_variant(pol.handle, 1)
+    obs = W.make_obs(spec, Bsz, seed=7)
+    out, _ = _check_forward(pol, qp, spec, obs, _edge_and_random_rows(Bsz, 256, 7), check_layers=True)
+    B.actorq_policy_set_fused_variant(pol.handle, 2)
+    other, _ = pol.forward(torch.from_numpy(obs).cuda())
+    torch.cuda.synchronize()
+    assert pol.status() == B.OK and torch.equal(out, other)
+    pol.close()

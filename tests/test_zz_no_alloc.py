@@ -1,4 +1,4 @@
-"""The allocation-free forward against the ordinary one, through the C ABI.
+"""The allocation-free forward against the ordinary one (and the CPU checker), through the C ABI.
 
 Some deployments cannot let the library allocate once the actor loop is live: the learner's
 framework already owns the device's memory pool, and a raw cudaMalloc both risks failing and stalls
@@ -16,6 +16,7 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
+from oracle import oracle as O                      # noqa: E402
 from paper_1910_01055_b200 import binding as B      # noqa: E402
 from paper_1910_01055_b200 import workloads as W    # noqa: E402
 
@@ -34,6 +35,12 @@ def _both(pol, spec, obs_np):
     assert np.all(np.abs(o - r) <= REL_TOL * np.abs(r) + 1e-30), float(np.abs(o - r).max())
     if ref_act is not None:
         assert torch.equal(act, ref_act)
+    # and against the CPU checker directly, so that this entry point does not lean on the other one
+    qp = O.quantize_policy(spec.layers, spec.input_ranges, spec.head, spec.obs_dtype)
+    y_ref, act_ref, _ = O.forward(qp, obs_np)
+    assert np.all(np.abs(o - y_ref) <= REL_TOL * np.abs(y_ref) + 1e-30), float(np.abs(o - y_ref).max())
+    if act_ref is not None:
+        assert np.array_equal(o, y_ref) and np.array_equal(act.cpu().numpy(), act_ref)
 
 
 @pytest.mark.parametrize("kind", ["mlp", "conv"])
