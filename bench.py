@@ -28,12 +28,42 @@ METRIC = "int8 policy inferences/sec"
 UNIT = "inferences/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_BF16 = 2.0     # nominal dense tensor ratio (4.5 POPS int8 vs 2.25 PFLOP/s bf16)
-# ncu capture of the forward kernel on mlp_wide: (dram bytes read + written, rows captured, bytes that
-# do not scale with the rows), see profiles/; None = not captured since the kernel last changed
-NCU_TRAFFIC_MLP_WIDE = (22.842624e6, 37888, 3.4e6)
-# actorq_2048: DRAM bytes of the four layer launches of one forward (rate x duration per launch,
-# profiles/fc_pair_kernel_actorq_2048_b65536.md), captured batch, weight images (read once per launch)
-NCU_TRAFFIC_ACTORQ_2048 = (717e6, 65536, 8.6e6)
+# DRAM traffic of the dominant forward kernel, from ncu captures summarised under profiles/ -- constants
+# taken from those captures, not measured by this run.  Per workload: kernel name, source file of the
+# kernel with the sha1 it had when the counters were taken (a changed file nulls the figure), dram
+# bytes read + written at the captured batch, captured batch, bytes that do not scale with the rows
+# (weight images, read from DRAM once per launch).
+NCU_TRAFFIC = {
+    "mlp_wide": ("fused_mlp_pair_kernel (forward)", "mlp_fused_pair.cu", "ec865bb3aaf97e9da53adecae889c597a8b8837a", 22.842624e6, 37888, 3.4e6),
+    "actorq_2048": ("fc_pair_kernel x layers (forward)", "fc_pair.cu", "2308d1a418591197491457222fe768ff86e5e879", 717e6, 65536, 8.6e6),
+}
+
+
+def ncu_traffic(workload: str, batch: int):
+    """(kernel name, bytes per launch or None, note) from the table above, scaled by rows."""
+    import hashlib
+    if workload not in NCU_TRAFFIC:
+        return None, None, "no ncu capture for this workload"
+    name, src, sha, cap_bytes, cap_rows, fixed = NCU_TRAFFIC[workload]
+    path = os.path.join(ROOT, "paper_1910_01055_b200", "csrc", src)
+    with open(path, "rb") as f:
+        now = hashlib.sha1(f.read()).hexdigest()
+    if now != sha:
+        return name, None, f"{src} changed since the ncu capture"
+    return name, (cap_bytes - fixed) * batch / float(cap_rows) + fixed, (
+        f"constant from the ncu capture at B={cap_rows} (profiles/), scaled by rows, {fixed / 1e6:.1f} MB of weight images counted once")
+
+
+def cpu_baseline_single_thread(workload: str, rows: int):
+    """The same checker run restricted to one thread (a child process with OMP_NUM_THREADS=1)."""
+    code = ("import sys, json; sys.path.insert(0, %r); import bench; from paper_1910_01055_b200 import workloads as W; "
+            "r, _ = bench.cpu_baseline(W.build_config(%r), %d); print(json.dumps(r))" % (ROOT, workload, rows))
+    env = dict(os.environ, OMP_NUM_THREADS="1", CUDA_VISIBLE_DEVICES="")
+    try:
+        res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+        return json.loads(res.stdout.strip().splitlines()[-1])
+    except Exception as e:      # the single-thread figure is an extra; its absence must not lose the bench line
+        return {"error": repr(e)}
 
 
 def load_peaks():
@@ -213,6 +243,41 @@ def run_quantizer_stream(args):
     pol.close()
 
 
+def measure_int8_peak(torch, B, pol, sustained_s: float = 1.0):
+    """The GPU's achieved dense INT8 tensor rate, measured in this process with the library's bare
+    tcgen05.mma kind::i8 loop (all SM pairs, operands resident, no epilogue): `burst` = best of 10
+    launches of about 2 ms, `sustained` = launches back to back for about `sustained_s` seconds (the
+    power cap then sets the clock).  Both operand placements are timed; the better one is the peak."""
+    stream = torch.cuda.current_stream()
+    res = {}
+    for name, in_tmem in (("a_smem", False), ("a_tmem", True)):
+        groups = 4096
+        ops = B.actorq_selftest_int8_mma_peak(pol.handle, groups, in_tmem)          # warm-up, also sizes the launch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream); ops = B.actorq_selftest_int8_mma_peak(pol.handle, groups, in_tmem); e1.record(stream)
+        torch.cuda.synchronize()
+        ms = max(e0.elapsed_time(e1), 1e-3)
+        groups = int(max(256, min(1 << 20, groups * 2.0 / ms)))                     # about 2 ms per launch
+        best = 0.0
+        for _ in range(10):
+            e0.record(stream); ops = B.actorq_selftest_int8_mma_peak(pol.handle, groups, in_tmem); e1.record(stream)
+            torch.cuda.synchronize()
+            best = max(best, ops / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+        n = max(1, int(sustained_s * 1e3 / 2.0))
+        e0.record(stream)
+        for _ in range(n):
+            ops = B.actorq_selftest_int8_mma_peak(pol.handle, groups, in_tmem)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        res[name] = {"burst": best, "sustained": n * ops / (e0.elapsed_time(e1) * 1e-3) / 1e12}
+    if pol.status() != B.OK:
+        return None
+    top = max(res.values(), key=lambda r: r["burst"])
+    return {"burst": top["burst"], "sustained": max(r["sustained"] for r in res.values()), "unit": "TOP/s",
+            "by_operand_placement": res,
+            "how": "tcgen05.mma.cta_group::2.kind::i8 M=256 n=256 K=32, one issuing thread per SM pair, no epilogue"}
+
+
 def bf16_comparator(torch, spec, layers_dev, obs_dev, reps=20):
     """The same network with bf16 weights / activations through torch's library kernels (cuBLAS / cuDNN)
     on the same GPU and batch: a comparator for the report, not part of the product."""
@@ -281,6 +346,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mlp_wide", choices=list(W.CONFIGS))
     ap.add_argument("--batch", type=int, default=0, help="rows per GPU per step (default: the config's batch)")
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="how many times the K-step region is timed (default: 5 up to 500 steps, 3 up to 1000, else 1); the median repeat is reported")
+    ap.add_argument("--no-int8-peak", action="store_true", help="skip the in-process measurement of the INT8 tensor peak")
     ap.add_argument("--ref-rows", type=int, default=2048)
     ap.add_argument("--cpu-rows", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -361,28 +429,38 @@ def main():
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    # the K-step region is timed `repeats` times (each bracketed by a barrier + synchronize); the
+    # reported figures are those of the median repeat, the spread is printed beside them
+    repeats = args.repeats or (5 if args.steps <= 500 else 3 if args.steps <= 1000 else 1)
+    runs = []
     launches = 0
-    outer = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    barrier()
-    outer[0].record(stream)
-    for i in range(args.steps):
-        ev[i][0].record(stream)
-        pol.quantize(layers_dev, spec.input_ranges)
-        lq = B.actorq_policy_last_launch_count(pol.handle)
-        ev[i][1].record(stream)
-        pol.forward(dev_obs[i % n_rot], out, actions)
-        ev[i][2].record(stream)
-        launches += lq + B.actorq_policy_last_launch_count(pol.handle)
-        if flush is not None:
-            flush.fill_(i & 0xff)
-    outer[1].record(stream)
-    barrier()
-    q_ms = np.array([ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)])
-    f_ms = np.array([ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)])
-    # device time of the K steps: the whole region, or (when an L2 flush runs between steps) the
-    # sum of the per-step spans, which leaves the flush writes out
-    step_ms = float(outer[0].elapsed_time(outer[1])) if flush is None else float((q_ms + f_ms).sum())
+    for rep in range(repeats):
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        outer = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        launches = 0
+        barrier()
+        outer[0].record(stream)
+        for i in range(args.steps):
+            ev[i][0].record(stream)
+            pol.quantize(layers_dev, spec.input_ranges)
+            lq = B.actorq_policy_last_launch_count(pol.handle)
+            ev[i][1].record(stream)
+            pol.forward(dev_obs[(rep * args.steps + i) % n_rot], out, actions)
+            ev[i][2].record(stream)
+            launches += lq + B.actorq_policy_last_launch_count(pol.handle)
+            if flush is not None:
+                flush.fill_(i & 0xff)
+        outer[1].record(stream)
+        barrier()
+        q = np.array([ev[i][0].elapsed_time(ev[i][1]) for i in range(args.steps)])
+        f = np.array([ev[i][1].elapsed_time(ev[i][2]) for i in range(args.steps)])
+        # device time of the K steps: the whole region, or (when an L2 flush runs between steps) the
+        # sum of the per-step spans, which leaves the flush writes out
+        region = float(outer[0].elapsed_time(outer[1])) if flush is None else float((q + f).sum())
+        runs.append((region, q, f))
+    order = sorted(range(repeats), key=lambda r: runs[r][0])
+    step_ms, q_ms, f_ms = runs[order[repeats // 2]]
+    region_all = [r[0] for r in runs]
 
     # end to end through the host-buffer call of the C ABI: pinned host observations in, outputs out,
     # chunked and pipelined inside the library; the re-quantize of the step goes first on the stream
@@ -415,30 +493,25 @@ def main():
         fwd_ms = float(np.mean(f_ms))
         achieved = ops_per_launch / (fwd_ms * 1e-3) / 1e12
         peak = INT8_OVER_BF16 * float(peaks["bf16_tflops"])
-        # DRAM traffic of the dominant kernel per launch, from one ncu capture of that kernel
-        # (profiles/): NCU_TRAFFIC holds (bytes read + written at the captured batch, captured batch).
-        # Traffic grows with the rows (observations in, outputs out) on top of the weight image,
-        # which is read from DRAM once, so it is scaled by rows to this batch.  None until the
-        # current kernel has been captured.
-        if args.workload == "mlp_wide":
-            kernel_name = "fused_mlp_pair_kernel (forward)"
-            if NCU_TRAFFIC_MLP_WIDE is not None:
-                cap_bytes, cap_rows, fixed = NCU_TRAFFIC_MLP_WIDE
-                traffic = (cap_bytes - fixed) * batch / float(cap_rows) + fixed
-                traffic_note = f"ncu dram bytes at B={cap_rows} scaled by rows (weight image {fixed / 1e6:.1f} MB counted once)"
-            else:
-                traffic, traffic_note = None, "kernel changed since the last ncu capture"
-        elif args.workload == "actorq_2048" and NCU_TRAFFIC_ACTORQ_2048 is not None:
-            kernel_name = "fc_pair_kernel x layers (forward)"
-            cap_bytes, cap_rows, fixed = NCU_TRAFFIC_ACTORQ_2048
-            traffic = (cap_bytes - fixed) * batch / float(cap_rows) + fixed
-            traffic_note = (f"ncu dram bytes of the four layer launches at B={cap_rows}, scaled by rows "
-                            f"(weight images {fixed / 1e6:.1f} MB counted once); activations between layers go through device memory")
-        else:
+        kernel_name, traffic, traffic_note = ncu_traffic(args.workload, batch)
+        if kernel_name is None:
             wide = max(l.out_features for l in spec.layers[:-1]) > 1024
-            kernel_name = ("conv_gemm_kernel x layers (forward)" if spec.obs_dtype != "f32" else
-                           "fc_pair_kernel x layers (forward)" if wide else "fused_mlp_pair_kernel (forward)")
-            traffic, traffic_note = None, "no ncu capture for this workload"
+            kernel_name = ("conv layer kernels (forward)" if spec.obs_dtype != "f32" else
+                           "fc_pair_kernel x layers (forward)" if wide else "fused MLP kernel (forward)")
+        # denominator: the INT8 tensor rate measured in this process by the library's bare MMA loop
+        # (burst: this bench times short regions); 2 x the measured bf16 figure only if that is skipped
+        int8_peak = None
+        if not args.no_int8_peak:
+            peak_sampler = ClockSampler(local)
+            peak_sampler.start()
+            int8_peak = measure_int8_peak(torch, B, pol)
+            peak_clocks = peak_sampler.stop()
+            if int8_peak is not None:
+                int8_peak["clocks"] = peak_clocks
+        if int8_peak is not None:
+            peak, peak_source = int8_peak["burst"], "measured int8 (bare tcgen05.mma kind::i8 loop, burst, this run)"
+        else:
+            peak_source = f"2 x bf16 burst of {peaks['_source']} ({peaks['bf16_tflops']} TFLOP/s)"
         result = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_ms / args.steps, "higher_is_better": True,
@@ -449,13 +522,18 @@ def main():
                               f"({n_rot * obs_bytes / 1e6:.0f} MB > 126 MB L2)" if flush is None
                               else "256 MB flush buffer written between timed steps"),
                        "quantize_ms": float(np.mean(q_ms)), "forward_ms": fwd_ms,
-                       "forward_ms_best": float(np.min(f_ms)), "device_status": status},
+                       "forward_ms_best": float(np.min(f_ms)), "device_status": status,
+                       "repeats": repeats, "timing": "median of the repeats of the K-step region",
+                       "region_ms_all_repeats": [round(x, 4) for x in region_all]},
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TOP/s",
                          "frac": achieved / peak, "traffic": traffic,
                          "traffic_note": traffic_note,
                          "kernel": kernel_name,
-                         "peak_source": f"2 x bf16 burst of {peaks['_source']} ({peaks['bf16_tflops']} TFLOP/s)",
-                         "frac_of_sustained": achieved / (INT8_OVER_BF16 * float(peaks["bf16_tflops_sustained"])),
+                         "peak_source": peak_source,
+                         "int8_peak_measured": int8_peak,
+                         "frac_of_measured_int8_sustained": (achieved / int8_peak["sustained"]) if int8_peak else None,
+                         "frac_of_2x_bf16": achieved / (INT8_OVER_BF16 * float(peaks["bf16_tflops"])),
+                         "frac_of_2x_bf16_sustained": achieved / (INT8_OVER_BF16 * float(peaks["bf16_tflops_sustained"])),
                          "frac_of_nominal_4500": achieved / 4500.0,
                          "ops_per_launch": ops_per_launch},
             "e2e": {"value": batch * world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
@@ -470,6 +548,7 @@ def main():
                                                     W.CONFIGS["actor_sweep"]["batches"] if spec.obs_dtype == "f32" else [1, 16, 256, 1024])
         if not args.no_cpu_baseline:
             result["cpu_baseline"], _ = cpu_baseline(spec, min(args.cpu_rows, batch))
+            result["cpu_baseline"]["single_thread"] = cpu_baseline_single_thread(args.workload, min(512, args.cpu_rows, batch))
             result["int8_vs_fp"] = int8_vs_fp(torch, pol, spec, min(512, batch))
         print(json.dumps(result))
     pol.close()

@@ -279,6 +279,18 @@ int actorq_policy_set_fused_variant(actorq_policy *policy, int variant);
  * (Diagnostics; the paper has no counterpart.) */
 int actorq_selftest_bounded_wait(actorq_policy *policy, long long limit_ns, void *cuda_stream);
 
+/* The GPU's achieved dense INT8 tensor-core rate, for roofline denominators: launches a kernel that
+ * only issues the instruction the layer kernels use (tcgen05.mma.cta_group::2.kind::i8, M = 256,
+ * n = 256, K = 32) on every SM pair -- operands resident in shared memory (a_in_tmem = 0; the two
+ * accumulators alternate) or the A operand in tensor memory (a_in_tmem = 1) -- with no epilogue and
+ * no memory traffic.  mma_groups (1 .. 2^24) = groups of four instructions per SM pair; *ops (host,
+ * may be NULL) receives the integer operations of the launch (2 per multiply-accumulate).  The
+ * caller times the launch with events on cuda_stream; rate = *ops / time.  The kernel's only wait is
+ * bounded (ACTORQ_ERR_TIMEOUT in the policy's status word); keep a launch to a few milliseconds.
+ * (Measurement aid; the paper has no counterpart.) */
+int actorq_selftest_int8_mma_peak(actorq_policy *policy, long long mma_groups, int a_in_tmem,
+                                  long long *ops, void *cuda_stream);
+
 /* Number of kernel launches the last actorq_policy_forward / actorq_quantize_params call on
  * this policy enqueued (for benchmark bookkeeping). */
 int actorq_policy_last_launch_count(const actorq_policy *policy);

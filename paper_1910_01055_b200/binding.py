@@ -25,7 +25,7 @@ NOALLOC_SCRATCH_BYTES = 64 << 20
 
 EXPORTS = ["actorq_policy_blob_bytes", "actorq_policy_export_blob", "actorq_policy_import_blob", "actorq_quantize_params", "actorq_policy_forward", "actorq_policy_forward_noalloc", "actorq_free", "actorq_policy_export_layer",
            "actorq_policy_forward_debug", "actorq_policy_last_device_status",
-           "actorq_policy_last_launch_count", "actorq_policy_timeout_info", "actorq_selftest_bounded_wait",
+           "actorq_policy_last_launch_count", "actorq_policy_timeout_info", "actorq_selftest_bounded_wait", "actorq_selftest_int8_mma_peak",
            "actorq_policy_set_fused_variant", "actorq_policy_forward_host", "actorq_policy_export_layer_channels", "actorq_policy_forward_explore", "actorq_version"]
 
 
@@ -258,6 +258,17 @@ def actorq_selftest_bounded_wait(policy: C.c_void_p, limit_ns: int, stream: Opti
     lib = load()
     lib.actorq_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_longlong, C.c_void_p]
     _check(lib.actorq_selftest_bounded_wait(policy, limit_ns, _stream_ptr(stream)), "actorq_selftest_bounded_wait")
+
+
+def actorq_selftest_int8_mma_peak(policy: C.c_void_p, mma_groups: int, a_in_tmem: bool = False,
+                                  stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Launch the bare int8 MMA loop (see actorq.h); returns the integer operations of the launch."""
+    lib = load()
+    lib.actorq_selftest_int8_mma_peak.argtypes = [C.c_void_p, C.c_longlong, C.c_int, C.POINTER(C.c_longlong), C.c_void_p]
+    ops = C.c_longlong(0)
+    _check(lib.actorq_selftest_int8_mma_peak(policy, mma_groups, int(a_in_tmem), C.byref(ops), _stream_ptr(stream)),
+           "actorq_selftest_int8_mma_peak")
+    return int(ops.value)
 
 
 def actorq_policy_set_fused_variant(policy: C.c_void_p, variant: int) -> None:

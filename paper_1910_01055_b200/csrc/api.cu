@@ -467,6 +467,11 @@ int actorq_selftest_bounded_wait(actorq_policy *p, long long limit_ns, void *cud
   return launch_selftest_bounded_wait(p, limit_ns, (cudaStream_t)cuda_stream);
 }
 
+int actorq_selftest_int8_mma_peak(actorq_policy *p, long long mma_groups, int a_in_tmem, long long *ops, void *cuda_stream) {
+  if (!p || mma_groups < 1 || mma_groups > (1ll << 24)) return ACTORQ_ERR_INVALID_ARG;
+  return launch_selftest_int8_mma_peak(p, mma_groups, a_in_tmem != 0, ops, (cudaStream_t)cuda_stream);
+}
+
 int actorq_policy_last_launch_count(const actorq_policy *p) { return p ? p->launches : 0; }
 
 const char *actorq_version(void) { return "actorq-b200 0.1 sm_100a"; }

@@ -127,6 +127,7 @@ int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, f
 // out[b][n] = clamp(out[b][n] + sigma[b] * noise[b][n], -1, 1) for the paths whose head does not do it
 int launch_explore(float *out, const float *sigma, const float *noise, long long batch, int out_dim, int sm_count, cudaStream_t st);
 int launch_selftest_bounded_wait(actorq_policy *p, long long limit_ns, cudaStream_t st);
+int launch_selftest_int8_mma_peak(actorq_policy *p, long long groups, int a_in_tmem, long long *ops, cudaStream_t st);
 // tcgen05 implicit-GEMM conv / FC layers (conv_gemm.cu)
 bool conv_gemm_supported(const actorq_policy *p);
 bool conv_gemm_image_perm(const actorq_policy *p, int l, int *C, int *KH, int *KW);
