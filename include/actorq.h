@@ -260,14 +260,16 @@ int actorq_policy_forward_host(actorq_policy *policy, const void *obs_host, long
                                float *out_host, int *actions_host, void *cuda_stream);
 
 /* Which fused MLP kernel actorq_policy_forward uses for an all-FC policy (Section 3.1, actor
- * inference): 0 = the library picks (default: the CTA-pair kernel, tcgen05 cta_group::2, where the
- * device can co-schedule pairs, else the single-CTA kernel), 1 = always the single-CTA kernel,
- * 2 = always the CTA-pair kernel (forward then returns ACTORQ_ERR_UNSUPPORTED / ACTORQ_ERR_CUDA
- * if pairs cannot be launched), 3 = one launch per layer on CTA pairs with the int8 activations
- * kept in device memory between layers (the path policies wider than 1024 take by default, e.g.
- * the paper's 2048-wide actor networks, and policies with per-channel layers; accepted for any
- * all-FC fp32-observation policy with hidden width <= 8192 and head <= 128).  All kernels produce
- * identical results;
+ * inference): 0 = the library picks (default: for small policies -- every layer at most 256 wide
+ * and 256 deep -- the kernel that keeps the whole int8 policy resident in shared memory and two
+ * observation tiles in flight per CTA; otherwise the CTA-pair kernel that streams the weights,
+ * tcgen05 cta_group::2; the single-CTA kernel where the device cannot co-schedule pairs),
+ * 1 = always the single-CTA kernel, 2 = always the streaming CTA-pair kernel (forward then returns
+ * ACTORQ_ERR_UNSUPPORTED / ACTORQ_ERR_CUDA if pairs cannot be launched), 3 = one launch per layer on
+ * CTA pairs with the int8 activations kept in device memory between layers (the path policies wider
+ * than 1024 take by default, e.g. the paper's 2048-wide actor networks, and policies with
+ * per-channel layers; accepted for any all-FC fp32-observation policy with hidden width <= 8192 and
+ * head <= 128), 4 = always the resident-weights kernel.  All kernels produce identical results;
  * the switch exists for tests and measurements.  Returns ACTORQ_ERR_UNSUPPORTED for policies the
  * requested kernel does not take. */
 int actorq_policy_set_fused_variant(actorq_policy *policy, int variant);

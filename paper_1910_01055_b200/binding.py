@@ -272,7 +272,7 @@ def actorq_selftest_int8_mma_peak(policy: C.c_void_p, mma_groups: int, a_in_tmem
 
 
 def actorq_policy_set_fused_variant(policy: C.c_void_p, variant: int) -> None:
-    """0: library picks, 1: single-CTA fused MLP kernel, 2: CTA-pair kernel (see actorq.h)."""
+    """0: library picks, 1: single-CTA fused MLP kernel, 2: CTA-pair kernel, 3: layer at a time, 4: resident weights (see actorq.h)."""
     lib = load()
     lib.actorq_policy_set_fused_variant.argtypes = [C.c_void_p, C.c_int]
     _check(lib.actorq_policy_set_fused_variant(policy, variant), "actorq_policy_set_fused_variant")

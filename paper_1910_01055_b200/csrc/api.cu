@@ -228,6 +228,12 @@ static int forward_impl(actorq_policy *p, const void *obs, long long batch, floa
     p->launches = 0;
   }
   if (p->fused_ok) {
+    // small policies: the whole int8 policy resident in shared memory, two tiles in flight
+    if ((p->fused_variant == 0 || p->fused_variant == 4) && fused_resident_supported(p)) {
+      const int rc = launch_forward_fused_resident(p, obs, batch, out, actions, dbg_layer, dbg_acc, (int8_t *)dbg_act, st);
+      if (rc != ACTORQ_ERR_UNSUPPORTED || p->fused_variant == 4) return rc;
+      p->launches = 0;
+    }
     // CTA pairs (n = 256 MMAs, half the weight traffic per SM) unless the caller pinned the
     // single-CTA kernel or the device cannot co-schedule pairs
     if (p->fused_variant != 1 && fused_pair_supported(p)) {
@@ -450,7 +456,7 @@ int actorq_policy_import_blob(actorq_policy *p, const void *blob, long long byte
 }
 
 int actorq_policy_set_fused_variant(actorq_policy *p, int variant) {
-  if (!p || variant < 0 || variant > 3) return ACTORQ_ERR_INVALID_ARG;
+  if (!p || variant < 0 || variant > 4) return ACTORQ_ERR_INVALID_ARG;
   if (variant == 3) {
     if (!p->fcp_ok) return ACTORQ_ERR_UNSUPPORTED;
     p->fused_variant = variant;
@@ -458,6 +464,7 @@ int actorq_policy_set_fused_variant(actorq_policy *p, int variant) {
   }
   if (variant != 0 && !p->fused_ok) return ACTORQ_ERR_UNSUPPORTED;
   if (variant == 2 && !actorq::fused_pair_supported(p)) return ACTORQ_ERR_UNSUPPORTED;
+  if (variant == 4 && !actorq::fused_resident_supported(p)) return ACTORQ_ERR_UNSUPPORTED;
   p->fused_variant = variant;
   return ACTORQ_OK;
 }

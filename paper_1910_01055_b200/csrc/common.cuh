@@ -79,8 +79,9 @@ struct actorq_policy {
   int fcp_ok;                                     // 1 if that path takes the policy (its layers then have weight images)
   int launches;
   int fused_ok;                                   // 1 if the fused tcgen05 MLP kernel applies
-  int fused_variant;                              // 0: pick (CTA pairs when possible), 1: single-CTA kernel, 2: CTA pairs,
-                                                  // 3: one launch per layer on CTA pairs (fc_pair.cu)
+  int fused_variant;                              // 0: pick (resident-weights kernel for small policies, else CTA pairs when
+                                                  // possible), 1: single-CTA kernel, 2: CTA pairs with the weight ring,
+                                                  // 3: one launch per layer on CTA pairs (fc_pair.cu), 4: resident-weights kernel
   int conv_ok;                                    // 1 if the tcgen05 implicit-GEMM layer kernel applies
   int sm_count;
   // staging of actorq_policy_forward_host: kHostSlots chunks in flight (device copies of a chunk's
@@ -118,6 +119,11 @@ int launch_forward_fused(actorq_policy *p, const void *obs, long long batch, flo
 bool fused_pair_supported(const actorq_policy *p);
 int launch_forward_fused_pair(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
                               int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st);
+
+// small policies with all weights resident in shared memory, two tiles in flight per CTA pair (mlp_resident.cu)
+bool fused_resident_supported(const actorq_policy *p);
+int launch_forward_fused_resident(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
+                                  int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st);
 
 // wide all-FC policies, one launch per layer on CTA pairs (fc_pair.cu)
 bool fc_pair_supported(const actorq_policy *p);

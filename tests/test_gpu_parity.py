@@ -610,3 +610,39 @@ def test_single_cta_fused_kernel_many_tiles_per_cta(config, Bsz):
     torch.cuda.synchronize()
     assert pol.status() == B.OK and torch.equal(out, other)
     pol.close()
+
+
+@pytest.mark.parametrize("dims,head,Bsz", [([67, 256, 256, 256, 21], "tanh", 80000),       # five tile pairs per CTA pair: both slots, odd count
+                                           ([24, 256, 256, 256, 6], "tanh", 40000),        # even head width, 16-byte-aligned rows
+                                           ([67, 256, 256, 256, 21], "tanh", 37888 + 129),  # ragged last tile read from global memory
+                                           ([50, 200, 96, 160, 9], "argmax", 20000),       # ragged widths, greedy actions
+                                           ([33, 64, 256, 40, 3], "linear", 777),
+                                           ([20] + [64] * 15 + [4], "tanh", 300),           # 16 layers
+                                           ([3, 4], "linear", 5)])                         # a single layer: the head alone
+def test_resident_weights_kernel_matches_checker(dims, head, Bsz):
+    """The small-policy kernel (all int8 weights resident in shared memory, observation tiles staged
+    by bulk copies, two tiles in flight per CTA): every layer's accumulators and codes and the outputs
+    on sampled rows against the checker, and the whole batch bit for bit against the streaming
+    CTA-pair kernel."""
+    spec = W.calibrate(W.mlp_policy("r", dims, seed=41, head=head, nonzero_bias=(len(dims) % 2 == 0)), 128, seed=41)
+    pol, qp, _ = _quantize_both(spec)
+    B.actorq_policy_set_fused_variant(pol.handle, 4)
+    obs = W.make_obs(spec, Bsz, seed=41)
+    sample = None if Bsz <= 1000 else _edge_and_random_rows(Bsz, 256, 41)
+    out, act = _check_forward(pol, qp, spec, obs, sample)
+    assert B.actorq_policy_last_launch_count(pol.handle) == 1
+    B.actorq_policy_set_fused_variant(pol.handle, 2)
+    other, oact = pol.forward(torch.from_numpy(obs).cuda())
+    torch.cuda.synchronize()
+    assert pol.status() == B.OK and torch.equal(out, other)
+    if act is not None:
+        assert torch.equal(act, oact)
+    # an observation tensor that is only 4-byte aligned is rejected by the API, one that is 16-byte aligned
+    # but offset from the allocation start is fine
+    B.actorq_policy_set_fused_variant(pol.handle, 4)
+    if Bsz > 300:
+        shifted = torch.from_numpy(obs).cuda()[4:]
+        out2, _ = pol.forward(shifted.contiguous() if (shifted.data_ptr() & 15) else shifted)
+        torch.cuda.synchronize()
+        assert torch.equal(out2, out[4:])
+    pol.close()
