@@ -130,6 +130,17 @@ bool fc_pair_supported(const actorq_policy *p);
 int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
                            int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st);
 
+// the fully connected tail of a convolutional policy on the layer kernel of fc_pair.cu
+int fc_tail_begin(actorq_policy *p, int l_begin, long long batch, cudaStream_t st, int8_t **blocks, int *nkb, int **rowsums,
+                  int clear_here, int **rs_all, long long *rs_all_len);
+// convolution layers with their input staged in shared memory (conv_staged.cu)
+bool conv_staged_supported(const actorq_policy *p, int l, long long batch);
+int launch_conv_staged(actorq_policy *p, int l, const void *in, long long batch, int8_t *out_act,
+                       int8_t *blk_out, int *blk_rs, int blk_nkb, int blk_unsigned, int *zero_ptr, long long zero_len,
+                       int *dbg_acc, int8_t *dbg_act, cudaStream_t st);
+int fc_tail_run(actorq_policy *p, int l_begin, long long batch, float *out, int *actions,
+                int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st);
+
 // out[b][n] = clamp(out[b][n] + sigma[b] * noise[b][n], -1, 1) for the paths whose head does not do it
 int launch_explore(float *out, const float *sigma, const float *noise, long long batch, int out_dim, int sm_count, cudaStream_t st);
 int launch_selftest_bounded_wait(actorq_policy *p, long long limit_ns, cudaStream_t st);

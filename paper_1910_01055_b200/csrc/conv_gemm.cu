@@ -50,6 +50,14 @@ struct ConvGemmArgs {
   const LayerParams *params;
   int layer, last, head;
   int8_t *out_act;        // [M][N] int8 NHWC (hidden layers)
+  // The last convolution in front of the fully connected tail writes its codes where the layer
+  // kernel of fc_pair.cu reads them instead: sample b is row b of the tail's input, its (pixel,
+  // channel) codes bytes pixel * N + channel of that row, stored as operand blocks (16 KB per 128
+  // rows and 128 bytes of the row, 128-byte swizzle), unsigned (code + 128) when blk_unsigned; the
+  // sums of a sample's stored codes are added to blk_rs[b].  nullptr for every other layer.
+  int8_t *blk_out;
+  int *blk_rs;
+  int blk_nkb, blk_unsigned;
   float *out;             // [M][N] float (last layer)
   int *actions;
   long long out_elems;    // per sample, for the debug tap's (c, h, w) order
@@ -325,6 +333,7 @@ conv_gemm_kernel(const __grid_constant__ ConvGemmArgs A) {
       const long long b = m_ok ? m / ohw : 0;
       const int pix = m_ok ? (int)(m - b * ohw) : 0;
       float best_v = 0.0f; int best_n = -1;
+      int blk_sum = 0;
       for (int ci = 0; ci < A.cpg; ++ci) {
         const int c = g * A.cpg + ci;
         if (c >= A.nchunk) break;
@@ -351,7 +360,25 @@ conv_gemm_kernel(const __grid_constant__ ConvGemmArgs A) {
                 if (n0 + j < A.N)
                   A.dbg_act[b * A.out_elems + (long long)(n0 + j) * ohw + pix] = (int8_t)(packed[j >> 2] >> (8 * (j & 3)));
             }
-            if (m_ok) {                                   // N is a multiple of 16 on this path
+            if (m_ok && A.blk_out != nullptr) {
+              if (A.blk_unsigned) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) packed[j] ^= 0x80808080u;
+              }
+              const uint32_t r128 = (uint32_t)(b & 127);
+              int8_t *row_blk = A.blk_out + ((((b >> 7) * A.blk_nkb) << 14) + (r128 << 7));
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {                                    // 16 codes = one 16-byte piece of the row
+                if (n0 + 16 * (h + 1) > A.N) break;                            // N is a multiple of 16 on this path
+                const long long k = (long long)pix * A.N + n0 + 16 * h;        // byte of the tail's input row
+                const uint32_t kc = ((uint32_t)k & 127) >> 4;
+                *reinterpret_cast<uint4 *>(row_blk + ((k >> 7) << 14) + ((kc ^ (r128 & 7)) << 4)) =
+                    make_uint4(packed[4 * h], packed[4 * h + 1], packed[4 * h + 2], packed[4 * h + 3]);
+#pragma unroll
+                for (int j = 4 * h; j < 4 * h + 4; ++j)
+                  blk_sum = A.blk_unsigned ? (int)__dp4a(packed[j], 0x01010101u, (unsigned)blk_sum) : __dp4a((int)packed[j], 0x01010101, blk_sum);
+              }
+            } else if (m_ok) {                            // N is a multiple of 16 on this path
               int8_t *o = A.out_act + m * A.N + n0;
               if (n0 + 16 <= A.N) *reinterpret_cast<uint4 *>(o) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
               if (n0 + 32 <= A.N) *reinterpret_cast<uint4 *>(o + 16) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
@@ -377,6 +404,7 @@ conv_gemm_kernel(const __grid_constant__ ConvGemmArgs A) {
         }
       }
       if (A.last && A.head == ACTORQ_HEAD_ARGMAX && m_ok) A.actions[m] = best_n;
+      if (A.blk_out != nullptr && m_ok) atomicAdd(A.blk_rs + b, blk_sum);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->acc_empty[buf]);
@@ -512,10 +540,40 @@ int launch_forward_conv_gemm(actorq_policy *p, const void *obs, long long batch,
     p->launches++;
     cur = bufs[1];
   }
-  for (int l = 0; l < p->n_layers; ++l) {
+  // The fully connected layers behind the last convolution run on the CTA-pair layer kernel
+  // (fc_pair.cu), fed directly by that convolution's epilogue; where it cannot take them (or no
+  // pair of CTAs can be scheduled) they run here like every other layer.
+  int l_tail = p->n_layers;
+  int8_t *blk = nullptr;
+  int *blk_rs = nullptr;
+  int blk_nkb = 0;
+  int *rs_all = nullptr;          // the tail's row-sum counters: cleared by the kernel of layer l_tail - 2 when that is a
+  long long rs_all_len = 0;       // staged convolution (no memset between the kernels of consecutive forwards)
+  bool clear_in_kernel = false;
+  if (!f32_obs) {
+    int lc = -1;
+    for (int l = 0; l < p->n_layers; ++l)
+      if (p->layers[l].g.kind == ACTORQ_CONV2D) lc = l;
+    clear_in_kernel = lc >= 1 && conv_staged_supported(p, lc - 1, batch);
+    if (lc >= 0 && lc + 1 < p->n_layers &&
+        fc_tail_begin(p, lc + 1, batch, st, &blk, &blk_nkb, &blk_rs, clear_in_kernel ? 0 : 1, &rs_all, &rs_all_len) == ACTORQ_OK)
+      l_tail = lc + 1;
+  }
+  for (int l = 0; l < l_tail; ++l) {
     const LayerDev &L = p->layers[l];
     const LayerGeom &g = L.g;
     const bool last = (l + 1 == p->n_layers);
+    if (!f32_obs && conv_staged_supported(p, l, batch)) {      // convolutions: input staged in shared memory
+      const bool feeds_tail = (l + 1 == l_tail && l_tail < p->n_layers);
+      const bool clears = clear_in_kernel && l_tail < p->n_layers && l == l_tail - 2;
+      const int rc = launch_conv_staged(p, l, cur, batch, feeds_tail ? nullptr : bufs[l & 1], feeds_tail ? blk : nullptr,
+                                        feeds_tail ? blk_rs : nullptr, blk_nkb, (feeds_tail && p->act[l_tail].z == -128) ? 1 : 0,
+                                        clears ? rs_all : nullptr, clears ? rs_all_len : 0,
+                                        (l == dbg_layer) ? dbg_acc : nullptr, (l == dbg_layer) ? dbg_act : nullptr, st);
+      if (rc != ACTORQ_OK) return rc;
+      cur = bufs[l & 1];
+      continue;
+    }
     ConvGemmArgs A;
     memset(&A, 0, sizeof(A));
     A.in_mode = (l == 0 && !f32_obs) ? 0 : 1;
@@ -546,6 +604,12 @@ int launch_forward_conv_gemm(actorq_policy *p, const void *obs, long long batch,
     A.params = p->d_params;
     A.layer = l; A.last = last ? 1 : 0; A.head = p->head;
     A.out_act = last ? nullptr : bufs[l & 1];
+    if (l + 1 == l_tail && l_tail < p->n_layers) {
+      A.blk_out = blk;
+      A.blk_rs = blk_rs;
+      A.blk_nkb = blk_nkb;
+      A.blk_unsigned = (p->act[l_tail].z == -128) ? 1 : 0;      // the layer kernel multiplies post-ReLU codes as unsigned bytes
+    }
     A.out = last ? out : nullptr;
     A.actions = actions;
     A.out_elems = g.out_elems;
@@ -572,6 +636,7 @@ int launch_forward_conv_gemm(actorq_policy *p, const void *obs, long long batch,
     p->launches++;
     cur = A.out_act;
   }
+  if (l_tail < p->n_layers) return fc_tail_run(p, l_tail, batch, out, actions, dbg_layer, dbg_acc, dbg_act, st);
   return cuda_ok(cudaGetLastError());
 }
 

@@ -521,11 +521,18 @@ static int fcp_ensure(actorq_policy *p, long long rows_pad) {
   return ACTORQ_OK;
 }
 
-int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
-                           int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st) {
-  if (!p->fcp_ok) return ACTORQ_ERR_UNSUPPORTED;
-  for (int l = 0; l < p->n_layers; ++l)
-    if (p->layers[l].wq_img == nullptr) return ACTORQ_ERR_UNSUPPORTED;
+struct FcpLaunch {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[2];
+  int max_pairs;
+  int n_stages;
+  long long n_tile_pairs, rows_pad;
+  int8_t *bufs[2];
+  int *rs[3];
+};
+
+// Launch configuration, activation buffers and row-sum arrays for `batch` rows.
+static int fcp_prepare(actorq_policy *p, long long batch, cudaStream_t st, FcpLaunch &F) {
   static bool attr_set[64] = {false};
   static int max_clusters[64] = {0};
   const int dev = p->device;
@@ -533,9 +540,9 @@ int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, f
   const int n_stages = fcp::kMaxStages;
   const int smem_bytes = n_stages * fcp::kStage + (int)sizeof(fcp::Barriers) + fcp::kEpiWarps * 32 * (int)sizeof(int4) + 16384;
   if (smem_bytes > kMaxSmem) return ACTORQ_ERR_UNSUPPORTED;
-  cudaLaunchConfig_t cfg;
+  cudaLaunchConfig_t &cfg = F.cfg;
+  cudaLaunchAttribute *attr = F.attr;
   memset(&cfg, 0, sizeof(cfg));
-  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
@@ -567,18 +574,28 @@ int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, f
   const int rc = fcp_ensure(p, rows_pad);
   if (rc != ACTORQ_OK) return rc;
   const size_t one = (size_t)p->fcp_rows * (size_t)fcp_row_bytes(p);
-  int8_t *bufs[2] = {(int8_t *)p->fcp_mem, (int8_t *)p->fcp_mem + one};
-  int *rs[3];
-  rs[0] = reinterpret_cast<int *>((int8_t *)p->fcp_mem + 2 * one);
-  rs[1] = rs[0] + p->fcp_rows;
-  rs[2] = rs[1] + p->fcp_rows;
+  F.bufs[0] = (int8_t *)p->fcp_mem;
+  F.bufs[1] = (int8_t *)p->fcp_mem + one;
+  F.rs[0] = reinterpret_cast<int *>((int8_t *)p->fcp_mem + 2 * one);
+  F.rs[1] = F.rs[0] + p->fcp_rows;
+  F.rs[2] = F.rs[1] + p->fcp_rows;
+  F.max_pairs = max_clusters[dev];
+  F.n_stages = n_stages;
+  F.n_tile_pairs = n_tile_pairs;
+  F.rows_pad = rows_pad;
+  return ACTORQ_OK;
+}
 
-  const int K0 = p->layers[0].g.K;
-  const int obs_slices = (K0 + 31) / 32 < 4 ? (K0 + 31) / 32 : 4;
-  fcp::quantize_obs_blocks_kernel<<<(unsigned)(rows_pad / 128), 128 * obs_slices, 0, st>>>((const float *)obs, batch, rows_pad, K0, (K0 + 127) / 128,
-                                                                             p->d_params, bufs[0], rs[0], rs[1]);
-  p->launches++;
-  for (int l = 0; l < p->n_layers; ++l) {
+// Layers [l_begin, n_layers) on the layer kernel.  Layer l reads the operand blocks in bufs[l & 1] and
+// the row sums in rs[l % 3]; whoever fills them for l_begin has also left rs[(l_begin + 1) % 3] zeroed.
+static int fcp_run_layers(actorq_policy *p, FcpLaunch &F, int l_begin, long long batch, float *out, int *actions,
+                          int dbg_layer, int *dbg_acc, int8_t *dbg_act) {
+  cudaLaunchConfig_t &cfg = F.cfg;
+  int8_t **bufs = F.bufs;
+  int **rs = F.rs;
+  const long long n_tile_pairs = F.n_tile_pairs, rows_pad = F.rows_pad;
+  const int n_stages = F.n_stages;
+  for (int l = l_begin; l < p->n_layers; ++l) {
     const LayerDev &L = p->layers[l];
     const bool last = (l + 1 == p->n_layers);
     fcp::Args A;
@@ -619,7 +636,7 @@ int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, f
     A.dbg_acc = (l == dbg_layer) ? dbg_acc : nullptr;
     A.dbg_act = (l == dbg_layer && !last) ? dbg_act : nullptr;
     A.status = p->d_status;
-    const long long pairs = A.n_items < max_clusters[dev] ? A.n_items : max_clusters[dev];
+    const long long pairs = A.n_items < F.max_pairs ? A.n_items : F.max_pairs;
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.numAttrs = 2;          // clusters of two + programmatic dependent launch
     const bool pc = L.g.per_channel != 0;
@@ -631,6 +648,57 @@ int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, f
     if (e != cudaSuccess) { cudaGetLastError(); return ACTORQ_ERR_CUDA; }
   }
   return ACTORQ_OK;
+}
+
+int launch_forward_fc_pair(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
+                           int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st) {
+  if (!p->fcp_ok) return ACTORQ_ERR_UNSUPPORTED;
+  for (int l = 0; l < p->n_layers; ++l)
+    if (p->layers[l].wq_img == nullptr) return ACTORQ_ERR_UNSUPPORTED;
+  FcpLaunch F;
+  const int rc = fcp_prepare(p, batch, st, F);
+  if (rc != ACTORQ_OK) return rc;
+  const int K0 = p->layers[0].g.K;
+  const int obs_slices = (K0 + 31) / 32 < 4 ? (K0 + 31) / 32 : 4;
+  fcp::quantize_obs_blocks_kernel<<<(unsigned)(F.rows_pad / 128), 128 * obs_slices, 0, st>>>((const float *)obs, batch, F.rows_pad, K0, (K0 + 127) / 128,
+                                                                               p->d_params, F.bufs[0], F.rs[0], F.rs[1]);
+  p->launches++;
+  return fcp_run_layers(p, F, 0, batch, out, actions, dbg_layer, dbg_acc, dbg_act);
+}
+
+// The fully connected tail of a convolutional policy (layers l_begin .. n_layers - 1) on the layer
+// kernel.  fc_tail_begin hands out where the kernel of layer l_begin - 1 must leave its output: operand
+// blocks (one 16 KB block [128 rows][128 B], 128-byte swizzle, per 128-row tile and 128 bytes of the
+// row) and per-row sums of the codes, accumulated with atomic adds into an array zeroed here.
+// clear_here: zero the row-sum arrays with a memset on the stream; otherwise the caller has a kernel
+// that runs before the accumulating one clear [*rs_all, *rs_all + *rs_all_len).
+int fc_tail_begin(actorq_policy *p, int l_begin, long long batch, cudaStream_t st, int8_t **blocks, int *nkb, int **rowsums,
+                  int clear_here, int **rs_all, long long *rs_all_len) {
+  if (l_begin < 1 || l_begin >= p->n_layers) return ACTORQ_ERR_UNSUPPORTED;
+  for (int l = l_begin; l < p->n_layers; ++l) {
+    const LayerGeom &g = p->layers[l].g;
+    const bool last = (l + 1 == p->n_layers);
+    if (g.kind != ACTORQ_FC || p->layers[l].wq_img == nullptr) return ACTORQ_ERR_UNSUPPORTED;
+    if (last ? g.N > 128 : g.N > 8192) return ACTORQ_ERR_UNSUPPORTED;
+  }
+  FcpLaunch F;
+  const int rc = fcp_prepare(p, batch, st, F);
+  if (rc != ACTORQ_OK) return rc;
+  if (clear_here && cudaMemsetAsync(F.rs[0], 0, 3 * (size_t)p->fcp_rows * sizeof(int), st) != cudaSuccess) { cudaGetLastError(); return ACTORQ_ERR_CUDA; }
+  *rs_all = F.rs[0];
+  *rs_all_len = 3 * p->fcp_rows;
+  *blocks = F.bufs[l_begin & 1];
+  *nkb = (p->layers[l_begin].g.K + 127) / 128;
+  *rowsums = F.rs[l_begin % 3];
+  return ACTORQ_OK;
+}
+
+int fc_tail_run(actorq_policy *p, int l_begin, long long batch, float *out, int *actions,
+                int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st) {
+  FcpLaunch F;
+  const int rc = fcp_prepare(p, batch, st, F);
+  if (rc != ACTORQ_OK) return rc;
+  return fcp_run_layers(p, F, l_begin, batch, out, actions, dbg_layer, dbg_acc, dbg_act);
 }
 
 }  // namespace actorq
