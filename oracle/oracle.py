@@ -353,3 +353,56 @@ def forward_f64(layers: Sequence, obs: np.ndarray, head: str, obs_dtype: str):
     if head == "tanh":
         x = np.tanh(x)
     return x, inputs
+
+
+# ---- counter-based exploration noise (Section 5, set-up: Gaussian noise on the actor's policy output) ------
+# The paper does not say how the actor draws its noise.  Reading taken here: row b, column n of a forward
+# call with seed s gets the standard normal z[b][n] of a counter-based generator, so that a row's noise does
+# not depend on the batch it travels in:
+#   (x0, x1, x2, x3) = Philox-4x32-10(counter = (b mod 2^32, b div 2^32, n div 4, 0), key = (s mod 2^32, s div 2^32))
+#   the pair (x0, x1) serves columns 4j, 4j + 1 and (x2, x3) columns 4j + 2, 4j + 3 of block j = n div 4:
+#   u1 = ((xa >> 8) + 1/2) 2^-24, u2 = ((xb >> 8) + 1/2) 2^-24            (both exactly representable in binary32)
+#   z_even = sqrt(-2 ln u1) cos(2 pi u2),  z_odd = sqrt(-2 ln u1) sin(2 pi u2)       (Box-Muller)
+# Philox-4x32-10 is the generator of Salmon, Moraes, Dror and Shaw, "Parallel random numbers: as easy as
+# 1, 2, 3" (SC'11), written out below from its definition; the checker evaluates the transform in double.
+
+_PHILOX_M0, _PHILOX_M1 = np.uint64(0xD2511F53), np.uint64(0xCD9E8D57)
+_PHILOX_W0, _PHILOX_W1 = np.uint64(0x9E3779B9), np.uint64(0xBB67AE85)
+_MASK32 = np.uint64(0xFFFFFFFF)
+
+
+def philox4x32_10(counter, key):
+    """counter: 4 arrays (or ints) of 32-bit words, key: 2 words; returns 4 uint64 arrays holding 32-bit words."""
+    c = [np.asarray(x, dtype=np.uint64) & _MASK32 for x in counter]
+    c = list(np.broadcast_arrays(*c))
+    k0, k1 = (np.uint64(int(key[0]) & 0xFFFFFFFF), np.uint64(int(key[1]) & 0xFFFFFFFF))
+    for _ in range(10):
+        p0 = _PHILOX_M0 * c[0]                 # 32 x 32 -> 64-bit products
+        p1 = _PHILOX_M1 * c[2]
+        hi0, lo0 = p0 >> np.uint64(32), p0 & _MASK32
+        hi1, lo1 = p1 >> np.uint64(32), p1 & _MASK32
+        c = [hi1 ^ c[1] ^ k0, lo1, hi0 ^ c[3] ^ k1, lo0]
+        k0 = (k0 + _PHILOX_W0) & _MASK32       # the key schedule: one Weyl step per round
+        k1 = (k1 + _PHILOX_W1) & _MASK32
+    return c
+
+
+def exploration_normals(seed: int, row0: int, rows: int, cols: int) -> np.ndarray:
+    """z[b][n] (float64) for rows row0 .. row0 + rows - 1 and columns 0 .. cols - 1 of a call with this seed."""
+    b = (np.arange(rows, dtype=np.uint64) + np.uint64(row0)).reshape(-1, 1)
+    n = np.arange(cols, dtype=np.uint64).reshape(1, -1)
+    x = philox4x32_10((b & _MASK32, b >> np.uint64(32), n >> np.uint64(2), np.uint64(0)), (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    second_pair = ((n >> np.uint64(1)) & np.uint64(1)) == 1
+    xa = np.where(second_pair, x[2], x[0])
+    xb = np.where(second_pair, x[3], x[1])
+    u1 = ((xa >> np.uint64(8)).astype(np.float64) + 0.5) * 2.0 ** -24
+    u2 = ((xb >> np.uint64(8)).astype(np.float64) + 0.5) * 2.0 ** -24
+    radius = np.sqrt(-2.0 * np.log(u1))
+    odd = (n & np.uint64(1)) == 1
+    return np.where(odd, radius * np.sin(2.0 * np.pi * u2), radius * np.cos(2.0 * np.pi * u2))
+
+
+def explore_seeded(y: np.ndarray, sigma: np.ndarray, seed: int, row0: int = 0) -> np.ndarray:
+    """explore() with the draws of exploration_normals, rounded to binary32 before the multiply."""
+    z = exploration_normals(seed, row0, y.shape[0], y.shape[1]).astype(np.float32)
+    return explore(y, sigma, z)

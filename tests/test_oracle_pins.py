@@ -595,3 +595,54 @@ def test_tiny_conv_policy_end_to_end(stride, per_channel):
                 eps = e + float(qp.layers[2].s_a) / 2
         assert np.all(np.abs(y_q[r].astype(np.float64) - y_fp[r]) <= e * (1 + 1e-6) + 1e-6), (r, y_q[r], y_fp[r], e)
     assert np.abs(y_q - y_fp).max() > 0
+
+
+# ---- counter-based exploration noise: Philox-4x32-10 + Box-Muller ------------------------------------
+
+def test_philox_known_answers():
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_known_answers.txt")
+    n = 0
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        c, k, want = [[int(w, 16) for w in part.split()] for part in line.split("|")]
+        got = [int(v) for v in O.philox4x32_10(c, k)]
+        assert got == want, (line, [hex(g) for g in got])
+        n += 1
+    assert n == 3
+    # vectorised over counters: the same words as one counter at a time
+    cs = np.array([[0, 1, 2, 3], [5, 0, 7, 0], [0xFFFFFFFF, 3, 0, 9]], dtype=np.uint64)
+    many = O.philox4x32_10([cs[:, i] for i in range(4)], (11, 12))
+    for r in range(3):
+        one = O.philox4x32_10([int(v) for v in cs[r]], (11, 12))
+        assert [int(m[r]) for m in many] == [int(v) for v in one]
+
+
+def test_exploration_normals_are_standard_normal_and_keyed_by_row_column_seed():
+    z = O.exploration_normals(1234, 0, 40000, 21)
+    assert z.shape == (40000, 21) and np.isfinite(z).all()
+    assert abs(z.mean()) < 4.0 / np.sqrt(z.size) and abs(z.var() - 1.0) < 0.01
+    assert abs((z ** 3).mean()) < 0.02 and abs((z ** 4).mean() - 3.0) < 0.05               # skewness 0, kurtosis 3
+    q = np.quantile(z, [0.001, 0.0228, 0.1587, 0.5, 0.8413, 0.9772, 0.999])
+    assert np.allclose(q, [-3.0902, -2.0, -1.0, 0.0, 1.0, 2.0, 3.0902], atol=0.03)          # the normal quantiles
+    assert np.abs(z).max() <= np.sqrt(-2.0 * np.log(0.5 * 2.0 ** -24)) + 1e-12             # largest radius the 24-bit uniform allows
+    # neighbouring columns (cos / sin of one pair, the two pairs of one counter) and rows are uncorrelated
+    for a, b in [(z[:, 0], z[:, 1]), (z[:, 0], z[:, 2]), (z[:, 3], z[:, 4]), (z[:-1, 5], z[1:, 5])]:
+        assert abs(np.corrcoef(a, b)[0, 1]) < 0.02
+    # a row's draws depend on (seed, absolute row, column) only: not on the batch or on how many columns are drawn
+    assert np.array_equal(O.exploration_normals(1234, 100, 7, 21), z[100:107])
+    assert np.array_equal(O.exploration_normals(1234, 0, 50, 6), z[:50, :6])
+    assert not np.array_equal(O.exploration_normals(1235, 0, 50, 6), z[:50, :6])
+    # rows beyond 2^32 use the second counter word
+    hi = O.exploration_normals(9, 2 ** 32 + 5, 2, 4)
+    assert not np.array_equal(hi, O.exploration_normals(9, 5, 2, 4))
+
+
+def test_explore_seeded_is_explore_with_those_draws():
+    rng = np.random.default_rng(5)
+    y = np.tanh(rng.standard_normal((64, 6))).astype(np.float32)
+    sigma = rng.uniform(0, 0.2, 64).astype(np.float32)
+    got = O.explore_seeded(y, sigma, 77, row0=3)
+    z = O.exploration_normals(77, 3, 64, 6).astype(np.float32)
+    assert np.array_equal(got, O.explore(y, sigma, z))
+    assert np.array_equal(O.explore_seeded(y, np.zeros(64, np.float32), 77), y)             # sigma 0: the policy's own action
