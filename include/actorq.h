@@ -237,6 +237,23 @@ int actorq_policy_forward_explore(actorq_policy *policy, const void *obs, long l
                                   const float *sigma, const float *noise, float *out, void *cuda_stream);
 
 /*
+ * The same with the noise drawn inside the library (the paper's actors draw their own noise; Section 5
+ * does not say how).  Row b, column n of the call gets the standard normal z of a counter-based
+ * generator keyed by (seed, first_row + b, n), so an actor's noise does not depend on the batch its
+ * observation travels in, and shards of one batch draw consistently when each passes its first row:
+ *   (x0..x3) = Philox-4x32-10(counter = (row mod 2^32, row div 2^32, n div 4, 0), key = (seed mod 2^32, seed div 2^32))
+ *   (x0, x1) serves columns 4j, 4j + 1 and (x2, x3) columns 4j + 2, 4j + 3 of block j = n div 4:
+ *   u1 = ((xa >> 9) + 1/2) 2^-23,  u2 = ((xb >> 9) + 1/2) 2^-23,
+ *   z = sqrt(-2 ln u1) cos(2 pi u2) for even n, ... sin(2 pi u2) for odd n            (Box-Muller)
+ *   out[b][n] = clamp(tanh(y[b][n]) + sigma[b] * z, -1, 1)
+ * The integer part is exact; the logarithm, square root and sine / cosine are single-precision
+ * library functions (a few ulp).  For policies the resident-weights kernel takes, the draw happens in
+ * that kernel's head; otherwise in one small kernel behind the forward.  ACTORQ_HEAD_TANH only.
+ */
+int actorq_policy_forward_explore_seeded(actorq_policy *policy, const void *obs, long long batch, const float *sigma,
+                                         unsigned long long seed, long long first_row, float *out, void *cuda_stream);
+
+/*
  * The same inference for callers whose observations live in HOST memory, as the paper's actors'
  * do (Section 3.1: actors run on CPU cores and feed the policy from their environments):
  *   obs_host      host; float [batch][obs_dim] or uint8 [batch][C][H][W]

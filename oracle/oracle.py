@@ -361,7 +361,7 @@ def forward_f64(layers: Sequence, obs: np.ndarray, head: str, obs_dtype: str):
 # not depend on the batch it travels in:
 #   (x0, x1, x2, x3) = Philox-4x32-10(counter = (b mod 2^32, b div 2^32, n div 4, 0), key = (s mod 2^32, s div 2^32))
 #   the pair (x0, x1) serves columns 4j, 4j + 1 and (x2, x3) columns 4j + 2, 4j + 3 of block j = n div 4:
-#   u1 = ((xa >> 8) + 1/2) 2^-24, u2 = ((xb >> 8) + 1/2) 2^-24            (both exactly representable in binary32)
+#   u1 = ((xa >> 9) + 1/2) 2^-23, u2 = ((xb >> 9) + 1/2) 2^-23            (24 significant bits: exact in binary32)
 #   z_even = sqrt(-2 ln u1) cos(2 pi u2),  z_odd = sqrt(-2 ln u1) sin(2 pi u2)       (Box-Muller)
 # Philox-4x32-10 is the generator of Salmon, Moraes, Dror and Shaw, "Parallel random numbers: as easy as
 # 1, 2, 3" (SC'11), written out below from its definition; the checker evaluates the transform in double.
@@ -395,8 +395,8 @@ def exploration_normals(seed: int, row0: int, rows: int, cols: int) -> np.ndarra
     second_pair = ((n >> np.uint64(1)) & np.uint64(1)) == 1
     xa = np.where(second_pair, x[2], x[0])
     xb = np.where(second_pair, x[3], x[1])
-    u1 = ((xa >> np.uint64(8)).astype(np.float64) + 0.5) * 2.0 ** -24
-    u2 = ((xb >> np.uint64(8)).astype(np.float64) + 0.5) * 2.0 ** -24
+    u1 = ((xa >> np.uint64(9)).astype(np.float64) + 0.5) * 2.0 ** -23
+    u2 = ((xb >> np.uint64(9)).astype(np.float64) + 0.5) * 2.0 ** -23
     radius = np.sqrt(-2.0 * np.log(u1))
     odd = (n & np.uint64(1)) == 1
     return np.where(odd, radius * np.sin(2.0 * np.pi * u2), radius * np.cos(2.0 * np.pi * u2))

@@ -26,7 +26,7 @@ NOALLOC_SCRATCH_BYTES = 64 << 20
 EXPORTS = ["actorq_policy_blob_bytes", "actorq_policy_export_blob", "actorq_policy_import_blob", "actorq_quantize_params", "actorq_policy_forward", "actorq_policy_forward_noalloc", "actorq_free", "actorq_policy_export_layer",
            "actorq_policy_forward_debug", "actorq_policy_last_device_status",
            "actorq_policy_last_launch_count", "actorq_policy_timeout_info", "actorq_selftest_bounded_wait", "actorq_selftest_int8_mma_peak",
-           "actorq_policy_set_fused_variant", "actorq_policy_forward_host", "actorq_policy_export_layer_channels", "actorq_policy_forward_explore", "actorq_version"]
+           "actorq_policy_set_fused_variant", "actorq_policy_forward_host", "actorq_policy_export_layer_channels", "actorq_policy_forward_explore", "actorq_policy_forward_explore_seeded", "actorq_version"]
 
 
 class LayerDesc(C.Structure):
@@ -145,6 +145,21 @@ def actorq_policy_forward_explore(policy: C.c_void_p, obs: torch.Tensor, sigma: 
     rc = lib.actorq_policy_forward_explore(policy, obs.data_ptr(), obs.shape[0], sigma.data_ptr(), noise.data_ptr(),
                                            out.data_ptr(), _stream_ptr(stream))
     _check(rc, "actorq_policy_forward_explore")
+
+
+def actorq_policy_forward_explore_seeded(policy: C.c_void_p, obs: torch.Tensor, sigma: torch.Tensor, seed: int, out: torch.Tensor,
+                                         first_row: int = 0, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """tanh policies: out = clamp(tanh(y) + sigma[row] * z, -1, 1) with z drawn by the library's counter-based
+    generator from (seed, first_row + row, column); see actorq.h."""
+    lib = load()
+    for t in (obs, sigma, out):
+        assert t.is_cuda and t.is_contiguous()
+    assert sigma.dtype == torch.float32 and out.dtype == torch.float32 and sigma.shape[0] == obs.shape[0]
+    lib.actorq_policy_forward_explore_seeded.argtypes = [C.c_void_p, C.c_void_p, C.c_longlong, C.c_void_p, C.c_ulonglong,
+                                                         C.c_longlong, C.c_void_p, C.c_void_p]
+    rc = lib.actorq_policy_forward_explore_seeded(policy, obs.data_ptr(), obs.shape[0], sigma.data_ptr(), seed, first_row,
+                                                  out.data_ptr(), _stream_ptr(stream))
+    _check(rc, "actorq_policy_forward_explore_seeded")
 
 
 def actorq_policy_forward_host(policy: C.c_void_p, obs: torch.Tensor, out: torch.Tensor,

@@ -270,6 +270,23 @@ int actorq_policy_forward_explore(actorq_policy *p, const void *obs, long long b
   return rc;
 }
 
+int actorq_policy_forward_explore_seeded(actorq_policy *p, const void *obs, long long batch, const float *sigma,
+                                         unsigned long long seed, long long first_row, float *out, void *cuda_stream) {
+  if (!p || batch < 0 || first_row < 0) return ACTORQ_ERR_INVALID_ARG;
+  if (p->head != ACTORQ_HEAD_TANH) return ACTORQ_ERR_UNSUPPORTED;
+  if (batch > 0 && !sigma) return ACTORQ_ERR_INVALID_ARG;
+  p->ex_sigma = sigma; p->ex_noise = nullptr; p->ex_applied = 0;
+  p->ex_seeded = 1; p->ex_seed = seed; p->ex_row0 = first_row;
+  int rc = forward_impl(p, obs, batch, out, nullptr, -1, nullptr, nullptr, cuda_stream);
+  const int applied = p->ex_applied;
+  p->ex_sigma = nullptr; p->ex_applied = 0; p->ex_seeded = 0;
+  if (rc != ACTORQ_OK || batch == 0 || applied) return rc;
+  rc = actorq::launch_explore_seeded(out, sigma, seed, first_row, batch, (int)p->layers[p->n_layers - 1].g.out_elems, p->sm_count,
+                                     (cudaStream_t)cuda_stream);
+  p->launches++;
+  return rc;
+}
+
 int actorq_policy_forward_debug(actorq_policy *policy, const void *obs, long long batch, float *out, int *actions,
                                 int layer, int *acc, signed char *act_q, void *cuda_stream) {
   if (!policy || layer < 0 || layer >= policy->n_layers || !acc) return ACTORQ_ERR_INVALID_ARG;

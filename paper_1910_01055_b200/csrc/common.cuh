@@ -99,6 +99,11 @@ struct actorq_policy {
   // draws [batch][out_dim]; a forward kernel that applies them in its head sets ex_applied
   const float *ex_sigma, *ex_noise;
   int ex_applied;
+  // actorq_policy_forward_explore_seeded: the draws come from the counter-based generator of
+  // explore_rng.cuh instead (ex_noise is then nullptr), keyed by ex_seed and the absolute row ex_row0 + b
+  int ex_seeded;
+  unsigned long long ex_seed;
+  long long ex_row0;
 };
 
 namespace actorq {
@@ -143,6 +148,8 @@ int fc_tail_run(actorq_policy *p, int l_begin, long long batch, float *out, int 
 
 // out[b][n] = clamp(out[b][n] + sigma[b] * noise[b][n], -1, 1) for the paths whose head does not do it
 int launch_explore(float *out, const float *sigma, const float *noise, long long batch, int out_dim, int sm_count, cudaStream_t st);
+int launch_explore_seeded(float *out, const float *sigma, unsigned long long seed, long long row0, long long batch, int out_dim,
+                          int sm_count, cudaStream_t st);
 int launch_selftest_bounded_wait(actorq_policy *p, long long limit_ns, cudaStream_t st);
 int launch_selftest_int8_mma_peak(actorq_policy *p, long long groups, int a_in_tmem, long long *ops, cudaStream_t st);
 // tcgen05 implicit-GEMM conv / FC layers (conv_gemm.cu)

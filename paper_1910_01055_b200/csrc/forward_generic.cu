@@ -6,6 +6,7 @@
 // Activations between layers are int8 codes in device scratch, [batch][features] with
 // convolutional features in (c, h, w) order.
 #include "common.cuh"
+#include "explore_rng.cuh"
 
 namespace actorq {
 
@@ -135,6 +136,26 @@ static int grid_for(long long work, int threads, int sm_count) {
   long long blocks = (work + threads - 1) / threads;
   long long cap = (long long)sm_count * 32;
   return (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
+}
+
+// the same with the draws of the counter-based generator (explore_rng.cuh), row = row0 + b
+__global__ void explore_seeded_kernel(float *__restrict__ out, const float *__restrict__ sigma, uint32_t seed_lo, uint32_t seed_hi,
+                                      long long row0, long long batch, int out_dim) {
+  const long long total = batch * out_dim;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long b = i / out_dim;
+    const int n = (int)(i - b * out_dim);
+    const float z = exploration_normal(seed_lo, seed_hi, row0 + b, n);
+    const float y = __fadd_rn(out[i], __fmul_rn(__ldg(sigma + b), z));
+    out[i] = fminf(fmaxf(y, -1.0f), 1.0f);
+  }
+}
+
+int launch_explore_seeded(float *out, const float *sigma, unsigned long long seed, long long row0, long long batch, int out_dim,
+                          int sm_count, cudaStream_t st) {
+  explore_seeded_kernel<<<grid_for(batch * out_dim, 256, sm_count), 256, 0, st>>>(out, sigma, (uint32_t)(seed & 0xffffffffull),
+                                                                                 (uint32_t)(seed >> 32), row0, batch, out_dim);
+  return cuda_ok(cudaGetLastError());
 }
 
 int launch_explore(float *out, const float *sigma, const float *noise, long long batch, int out_dim, int sm_count, cudaStream_t st) {

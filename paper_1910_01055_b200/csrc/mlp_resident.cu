@@ -27,6 +27,7 @@
 // abort flags, and both CTAs meet in a cluster barrier before tensor memory is released.
 #include <new>
 #include "tcgen05.cuh"
+#include "explore_rng.cuh"
 
 namespace actorq {
 
@@ -64,7 +65,10 @@ struct Args {
   float *out;
   int *actions;
   const float *sigma;      // exploration noise (tanh heads) or nullptr
-  const float *noise;
+  const float *noise;      // the caller's standard normal draws, or nullptr with noise_seeded: counter-based draws
+  int noise_seeded;
+  uint32_t seed_lo, seed_hi;
+  long long noise_row0;    // absolute row of the call's first observation
   int head;
   float obs_inv_s;         // input quantizer of the observations (host-known: 1 / s_a and z_a of layer 0)
   int obs_z;
@@ -531,11 +535,15 @@ fused_mlp_resident_kernel(const __grid_constant__ Args A) {
               if (A.head == ACTORQ_HEAD_TANH) {
                 y0 = tanhf(y0);
                 y1 = tanhf(y1);
-                if (A.noise != nullptr) {          // actor exploration: y + sigma * eps, kept in [-1, 1]
-                  y0 = __fadd_rn(y0, __fmul_rn(__ldg(A.sigma + q_row0 + r0), __ldg(A.noise + q_row0 * N + i0)));
+                if (A.noise != nullptr || A.noise_seeded) {          // actor exploration: y + sigma * eps, kept in [-1, 1]
+                  const float e0 = A.noise_seeded ? exploration_normal(A.seed_lo, A.seed_hi, A.noise_row0 + q_row0 + r0, i0 - r0 * N)
+                                                  : __ldg(A.noise + q_row0 * N + i0);
+                  y0 = __fadd_rn(y0, __fmul_rn(__ldg(A.sigma + q_row0 + r0), e0));
                   y0 = fminf(fmaxf(y0, -1.0f), 1.0f);
                   if (i1 < total) {
-                    y1 = __fadd_rn(y1, __fmul_rn(__ldg(A.sigma + q_row0 + r1), __ldg(A.noise + q_row0 * N + i1)));
+                    const float e1 = A.noise_seeded ? exploration_normal(A.seed_lo, A.seed_hi, A.noise_row0 + q_row0 + r1, i1 - r1 * N)
+                                                    : __ldg(A.noise + q_row0 * N + i1);
+                    y1 = __fadd_rn(y1, __fmul_rn(__ldg(A.sigma + q_row0 + r1), e1));
                     y1 = fminf(fmaxf(y1, -1.0f), 1.0f);
                   }
                 }
@@ -666,9 +674,13 @@ int launch_forward_fused_resident(actorq_policy *p, const void *obs, long long b
   A.out = out;
   A.actions = actions;
   A.head = p->head;
-  if (p->ex_noise != nullptr && p->head == ACTORQ_HEAD_TANH && dbg_layer < 0) {
+  if ((p->ex_noise != nullptr || p->ex_seeded) && p->head == ACTORQ_HEAD_TANH && dbg_layer < 0) {
     A.sigma = p->ex_sigma;
     A.noise = p->ex_noise;
+    A.noise_seeded = p->ex_seeded;
+    A.seed_lo = (uint32_t)(p->ex_seed & 0xffffffffull);
+    A.seed_hi = (uint32_t)(p->ex_seed >> 32);
+    A.noise_row0 = p->ex_row0;
     p->ex_applied = 1;
   }
   A.obs_dim = p->layers[0].g.K;

@@ -646,3 +646,38 @@ def test_resident_weights_kernel_matches_checker(dims, head, Bsz):
         torch.cuda.synchronize()
         assert torch.equal(out2, out[4:])
     pol.close()
+
+
+@pytest.mark.parametrize("dims,Bsz", [([67, 256, 256, 256, 21], 3000), ([24, 256, 256, 256, 6], 130),   # drawn in the resident kernel's head
+                                      ([128, 1024, 1024, 12], 513), ([10, 2048, 2048, 4], 70)])          # drawn by the kernel behind the forward
+def test_seeded_exploration_noise(dims, Bsz):
+    """actorq_policy_forward_explore_seeded against the checker's Philox-4x32-10 + Box-Muller draws.  The
+    integer part of the generator is exact on both sides; the normal transform runs in single precision on
+    the GPU (logarithm, square root, sine / cosine: a few ulp each, |z| <= 5.7) and in double in the checker,
+    so sigma * z may differ by 0.2 * 5.7 * 1e-6; on top of that the 1e-5 relative tolerance of tanh."""
+    spec = W.calibrate(W.mlp_policy("es", dims, seed=63, head="tanh"), 64, seed=63)
+    pol, qp, _ = _quantize_both(spec)
+    obs = W.make_obs(spec, Bsz, seed=63)
+    sigma = np.random.default_rng(63).uniform(0.0, 0.2, Bsz).astype(np.float32)
+    sigma[0] = 0.0
+    seed, first_row = 0x1234_5678_9ABC_DEF0, 2 ** 32 - 7                   # rows straddle the second counter word
+    out = torch.empty((Bsz, dims[-1]), dtype=torch.float32, device="cuda")
+    obs_d, sigma_d = torch.from_numpy(obs).cuda(), torch.from_numpy(sigma).cuda()
+    B.actorq_policy_forward_explore_seeded(pol.handle, obs_d, sigma_d, seed, out, first_row=first_row)
+    plain, _ = pol.forward(obs_d)
+    torch.cuda.synchronize()
+    assert pol.status() == B.OK
+    y_ref, _, _ = O.forward(qp, obs)
+    want = O.explore_seeded(y_ref, sigma, seed, row0=first_row)
+    got = out.cpu().numpy()
+    tol = REL_TOL * np.abs(y_ref) + 2.0e-6
+    assert np.all(np.abs(got - want) <= tol), float(np.abs(got - want).max())
+    assert np.array_equal(got[0], plain.cpu().numpy()[0])                  # sigma 0: the policy's own action
+    assert np.abs(got - plain.cpu().numpy()).max() > 0.05                  # and the noise is really there
+    # a row's noise does not depend on the batch: the second half alone, with its own first row
+    h = Bsz // 2
+    out2 = torch.empty((Bsz - h, dims[-1]), dtype=torch.float32, device="cuda")
+    B.actorq_policy_forward_explore_seeded(pol.handle, obs_d[h:].clone(), sigma_d[h:].clone(), seed, out2, first_row=first_row + h)
+    torch.cuda.synchronize()
+    assert torch.equal(out2, out[h:])
+    pol.close()

@@ -625,7 +625,7 @@ def test_exploration_normals_are_standard_normal_and_keyed_by_row_column_seed():
     assert abs((z ** 3).mean()) < 0.02 and abs((z ** 4).mean() - 3.0) < 0.05               # skewness 0, kurtosis 3
     q = np.quantile(z, [0.001, 0.0228, 0.1587, 0.5, 0.8413, 0.9772, 0.999])
     assert np.allclose(q, [-3.0902, -2.0, -1.0, 0.0, 1.0, 2.0, 3.0902], atol=0.03)          # the normal quantiles
-    assert np.abs(z).max() <= np.sqrt(-2.0 * np.log(0.5 * 2.0 ** -24)) + 1e-12             # largest radius the 24-bit uniform allows
+    assert np.abs(z).max() <= np.sqrt(-2.0 * np.log(0.5 * 2.0 ** -23)) + 1e-12             # largest radius the 23-bit uniform allows
     # neighbouring columns (cos / sin of one pair, the two pairs of one counter) and rows are uncorrelated
     for a, b in [(z[:, 0], z[:, 1]), (z[:, 0], z[:, 2]), (z[:, 3], z[:, 4]), (z[:-1, 5], z[1:, 5])]:
         assert abs(np.corrcoef(a, b)[0, 1]) < 0.02
