@@ -406,3 +406,42 @@ def explore_seeded(y: np.ndarray, sigma: np.ndarray, seed: int, row0: int = 0) -
     """explore() with the draws of exploration_normals, rounded to binary32 before the multiply."""
     z = exploration_normals(seed, row0, y.shape[0], y.shape[1]).astype(np.float32)
     return explore(y, sigma, z)
+
+
+# ---- the fp16 actor (Section 3.2: policies are quantized "to fp16 and int8"; the q = 16 rows of the
+# communication-vs-computation study) ---------------------------------------------------------------
+# Reading (the paper names the precision, not the arithmetic): weights and observations are rounded to
+# binary16 (round to nearest even); a layer is y[n] = sum_k a[k] w[n][k] + b[n] with the bias kept in
+# binary32; hidden layers apply ReLU and round the result to binary16 for the next layer; the head
+# applies tanh (or nothing).  A product of two binary16 numbers is exact in binary32 and in binary64,
+# so the checker forms the sum in binary64 (exact to ~1e-16 relative of the sum of magnitudes) and rounds
+# ONCE; an implementation that accumulates in binary32 differs by its accumulation error and, where that
+# moves a value across a rounding boundary, by one binary16 step (see the tolerance in the parity test).
+
+def cast_fp16(w: np.ndarray) -> np.ndarray:
+    """round to nearest even binary16 (values beyond 65504 become +-inf, as the format prescribes)"""
+    return np.asarray(w, dtype=np.float32).astype(np.float16)
+
+
+def forward_fp16(layers: Sequence, obs: np.ndarray, head: str):
+    """Returns (out float32 [B][out_dim], actions or None, trace) with trace[i] = layer i's binary16 output
+    activations (hidden layers) or its binary32 pre-activation (last layer)."""
+    a = cast_fp16(obs).astype(np.float64)
+    trace = []
+    n = len(layers)
+    y = None
+    for i, l in enumerate(layers):
+        w16 = cast_fp16(l.weight).astype(np.float64)
+        acc = a.reshape(a.shape[0], -1) @ w16.T
+        if l.bias is not None:
+            acc = acc + np.asarray(l.bias, dtype=np.float32).astype(np.float64)
+        if i + 1 < n:
+            h = np.maximum(acc, 0.0).astype(np.float16)          # one rounding of the (to 1e-16) exact value
+            trace.append(h)
+            a = h.astype(np.float64)
+        else:
+            pre = acc.astype(np.float32)
+            trace.append(pre)
+            y = np.tanh(acc).astype(np.float32) if head == "tanh" else pre
+    actions = argmax(y) if head == "argmax" else None
+    return y, actions, trace

@@ -646,3 +646,73 @@ def test_explore_seeded_is_explore_with_those_draws():
     z = O.exploration_normals(77, 3, 64, 6).astype(np.float32)
     assert np.array_equal(got, O.explore(y, sigma, z))
     assert np.array_equal(O.explore_seeded(y, np.zeros(64, np.float32), 77), y)             # sigma 0: the policy's own action
+
+
+# ---- the fp16 actor ------------------------------------------------------------------------------------
+
+def _rne_binary16(fr: F) -> F:
+    """correctly rounded binary16 (normal range) of an exact rational, independent of numpy's cast"""
+    if fr == 0:
+        return F(0)
+    sign = -1 if fr < 0 else 1
+    a = abs(fr)
+    e = math.floor(math.log2(a))
+    while F(2) ** e > a:
+        e -= 1
+    while F(2) ** (e + 1) <= a:
+        e += 1
+    e = max(e, -14)                                   # subnormals share the smallest normal exponent
+    ulp = F(2) ** (e - 10)
+    return sign * _rne(a / ulp) * ulp
+
+
+def test_fp16_cast_is_round_to_nearest_even():
+    rng = np.random.default_rng(70)
+    w = np.concatenate([rng.standard_normal(200) * 10.0 ** rng.uniform(-4, 3, 200),
+                        [1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 2049.0, 2051.0, 6.0e-8, 65504.0]]).astype(np.float32)   # ties and a subnormal
+    got = O.cast_fp16(w)
+    for x, g in zip(w.tolist(), got.tolist()):
+        assert F(g) == _rne_binary16(F(x)), (x, g)
+    rel = np.abs(got.astype(np.float64) - w.astype(np.float64)) / np.abs(w.astype(np.float64))
+    assert rel[np.abs(w) > 1e-4].max() <= 2.0 ** -11
+
+
+def test_fp16_forward_is_exact_on_a_power_of_two_grid():
+    """Small integers times powers of two: every product and sum is exact in binary16 / 32 / 64, so the fp16
+    forward must equal integer arithmetic exactly (a dropped bias, a transposed weight or a missing ReLU fails)."""
+    rng = np.random.default_rng(71)
+    w0 = rng.integers(-4, 5, (6, 5)).astype(np.float32) * 0.25
+    b0 = rng.integers(-3, 4, 6).astype(np.float32) * 0.5
+    w1 = rng.integers(-4, 5, (3, 6)).astype(np.float32) * 0.5
+    obs = rng.integers(-8, 9, (11, 5)).astype(np.float32) * 0.125
+    y, act, trace = O.forward_fp16([_L(w0, b0), _L(w1, None)], obs, "argmax")
+    h = np.maximum(obs.astype(np.float64) @ w0.astype(np.float64).T + b0, 0.0)
+    assert np.array_equal(trace[0].astype(np.float64), h)
+    assert np.array_equal(y.astype(np.float64), h @ w1.astype(np.float64).T)
+    assert np.array_equal(act, np.argmax(y, axis=1))
+
+
+@pytest.mark.parametrize("dims,head", [([3, 4, 2], "tanh"), ([5, 16, 8, 3], "linear")])
+def test_fp16_forward_close_to_fp_forward(dims, head):
+    """|y16 - y| within the bound propagated from one binary16 rounding (relative 2^-11) per weight, input
+    and hidden activation; and not vacuous: fp16 really differs from the un-rounded network."""
+    rng = np.random.default_rng(72)
+    layers = [_L((rng.standard_normal((dims[i + 1], dims[i])) * dims[i] ** -0.5).astype(np.float32),
+                 (rng.standard_normal(dims[i + 1]) * 0.1).astype(np.float32)) for i in range(len(dims) - 1)]
+    obs = rng.standard_normal((200, dims[0])).astype(np.float32)
+    y16, _, _ = O.forward_fp16(layers, obs, head)
+    y64, _ = O.forward_f64(layers, obs, head, "f32")
+    u = 2.0 ** -11
+    for r in range(obs.shape[0]):
+        a = np.abs(obs[r].astype(np.float64))
+        eps = a * u
+        x = obs[r].astype(np.float64)
+        for i, l in enumerate(layers):
+            Wm = l.weight.astype(np.float64)
+            e = np.abs(Wm) @ eps + (np.abs(Wm) * u) @ (np.abs(x) + eps)
+            pre = Wm @ x + l.bias.astype(np.float64)
+            if i + 1 < len(layers):
+                x = np.maximum(pre, 0)
+                eps = e + (np.abs(x) + e) * u
+        assert np.all(np.abs(y16[r].astype(np.float64) - y64[r]) <= e * (1 + 1e-6) + 1e-7), (r, y16[r], y64[r], e)
+    assert np.abs(y16 - y64).max() > 0
