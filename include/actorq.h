@@ -117,6 +117,26 @@ int actorq_quantize_params(const actorq_layer_desc *layers, int n_layers,
                            void *cuda_stream, actorq_policy **inout_policy);
 
 /*
+ * The fp16 actor (Section 3.2: policies are quantized "to fp16 and int8"; Section 5 runs actors and
+ * communication at q = 16 as well).  Casts the fp32 policy to binary16 instead of quantizing it to int8:
+ * every weight is rounded to nearest even binary16, biases stay binary32.  The resulting policy is used
+ * through actorq_policy_forward (also the host-buffer and exploration forms) and computes
+ *   layer:  y[n] = sum_k a[k] w[n][k] + b[n]   binary16 operands, binary32 accumulation on the tensor cores
+ *   hidden: a_next = round_to_binary16(max(y, 0));   last: out = tanh(y) or y, greedy action as for int8
+ * with the observations rounded to binary16 on the way in.  Results agree with a reference that sums in
+ * double and rounds once to within the accumulation error of binary32 plus, rarely, one binary16 step of a
+ * hidden activation (no bit-exact contract: the tensor core's summation order is not specified).
+ *   layers / head / obs_dtype / inout_policy   as for actorq_quantize_params (no activation ranges);
+ *                 *inout_policy != NULL must be a policy created by this call with the same architecture:
+ *                 it is re-cast in place without allocation or host synchronisation (the per-broadcast path).
+ * All-FC policies on float observations, every layer at most 8192 wide, the last at most 128:
+ * ACTORQ_ERR_UNSUPPORTED otherwise.  The inspection calls for int8 policies (export_layer, forward_debug,
+ * blobs, set_fused_variant, forward_noalloc) return ACTORQ_ERR_UNSUPPORTED for such a policy.
+ */
+int actorq_cast_params_fp16(const actorq_layer_desc *layers, int n_layers, int head, int obs_dtype,
+                            void *cuda_stream, actorq_policy **inout_policy);
+
+/*
  * Actor policy inference with the quantized policy (Section 3.1: the actors run the
  * quantized policy; Section 3.2: weights and activations in the same precision),
  * batched over `batch` independent observations.

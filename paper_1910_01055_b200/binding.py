@@ -26,7 +26,7 @@ NOALLOC_SCRATCH_BYTES = 64 << 20
 EXPORTS = ["actorq_policy_blob_bytes", "actorq_policy_export_blob", "actorq_policy_import_blob", "actorq_quantize_params", "actorq_policy_forward", "actorq_policy_forward_noalloc", "actorq_free", "actorq_policy_export_layer",
            "actorq_policy_forward_debug", "actorq_policy_last_device_status",
            "actorq_policy_last_launch_count", "actorq_policy_timeout_info", "actorq_selftest_bounded_wait", "actorq_selftest_int8_mma_peak",
-           "actorq_policy_set_fused_variant", "actorq_policy_forward_host", "actorq_policy_export_layer_channels", "actorq_policy_forward_explore", "actorq_policy_forward_explore_seeded", "actorq_version"]
+           "actorq_policy_set_fused_variant", "actorq_policy_forward_host", "actorq_policy_export_layer_channels", "actorq_policy_forward_explore", "actorq_policy_forward_explore_seeded", "actorq_cast_params_fp16", "actorq_version"]
 
 
 class LayerDesc(C.Structure):
@@ -131,6 +131,27 @@ def actorq_policy_forward(policy: C.c_void_p, obs: torch.Tensor, out: torch.Tens
     rc = lib.actorq_policy_forward(policy, obs.data_ptr(), obs.shape[0], out.data_ptr(),
                                    actions.data_ptr() if actions is not None else None, _stream_ptr(stream))
     _check(rc, "actorq_policy_forward")
+
+
+def actorq_cast_params_fp16(layers: Sequence[dict], head: str, obs_dtype: str, policy: Optional[C.c_void_p] = None,
+                            stream: Optional[torch.cuda.Stream] = None) -> C.c_void_p:
+    """Cast the fp32 policy to binary16 (the paper's q = 16 actor); returns the (new or re-cast) policy handle."""
+    lib = load()
+    n = len(layers)
+    descs = (LayerDesc * n)()
+    for i, l in enumerate(layers):
+        w = l["weight"]
+        assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
+        assert w.dim() == 2, "the fp16 actor takes fully connected layers"
+        b = l.get("bias")
+        descs[i].kind = FC
+        descs[i].out_features, descs[i].in_features = w.shape
+        descs[i].weight = w.data_ptr()
+        descs[i].bias = b.data_ptr() if b is not None else None
+    handle = policy if policy is not None else C.c_void_p(None)
+    lib.actorq_cast_params_fp16.argtypes = [C.POINTER(LayerDesc), C.c_int, C.c_int, C.c_int, C.c_void_p, C.POINTER(C.c_void_p)]
+    _check(lib.actorq_cast_params_fp16(descs, n, HEAD[head], OBS[obs_dtype], _stream_ptr(stream), C.byref(handle)), "actorq_cast_params_fp16")
+    return handle
 
 
 def actorq_policy_forward_explore(policy: C.c_void_p, obs: torch.Tensor, sigma: torch.Tensor, noise: torch.Tensor,

@@ -8,7 +8,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libactorq.so")
-SOURCES = ["api.cu", "quantize.cu", "forward_generic.cu", "mlp_fused.cu", "mlp_fused_pair.cu", "mlp_resident.cu", "fc_pair.cu", "conv_gemm.cu", "conv_staged.cu", "selftest_peak.cu"]
+SOURCES = ["api.cu", "quantize.cu", "forward_generic.cu", "mlp_fused.cu", "mlp_fused_pair.cu", "mlp_resident.cu", "fc_pair.cu", "fp16_pair.cu", "conv_gemm.cu", "conv_staged.cu", "selftest_peak.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--fmad=true", "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v"]
 

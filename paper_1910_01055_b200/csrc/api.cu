@@ -177,6 +177,7 @@ int actorq_quantize_params(const actorq_layer_desc *layers, int n_layers, const 
     if (isinf(input_ranges[l].min) || isinf(input_ranges[l].max)) return ACTORQ_ERR_INVALID_ARG;
   }
   actorq_policy *p = *inout_policy;
+  if (p != nullptr && p->precision == 16) return ACTORQ_ERR_INVALID_ARG;      // a policy cast to binary16 is re-cast, not quantized
   if (p == nullptr) {
     int rc = create_policy(layers, n_layers, head, obs_dtype, &p);
     if (rc != ACTORQ_OK) return rc;
@@ -220,6 +221,10 @@ static int forward_impl(actorq_policy *p, const void *obs, long long batch, floa
   if (p->head == ACTORQ_HEAD_ARGMAX && !actions) return ACTORQ_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(obs) & 15) != 0) return ACTORQ_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (p->precision == 16) {             // a policy cast to binary16: its own layer kernel, no debug taps
+    if (dbg_layer >= 0) return ACTORQ_ERR_UNSUPPORTED;
+    return launch_forward_fp16(p, obs, batch, out, actions, st);
+  }
   // Wide all-FC policies (and any all-FC policy when the caller asks for it): one launch per layer
   // on CTA pairs, activations as MMA operand blocks in device memory.
   if ((p->fused_variant == 3 || !p->fused_ok) && p->fcp_ok) {
@@ -248,6 +253,51 @@ static int forward_impl(actorq_policy *p, const void *obs, long long batch, floa
   if (p->conv_ok)
     return launch_forward_conv_gemm(p, obs, batch, out, actions, dbg_layer, dbg_acc, (int8_t *)dbg_act, st);
   return launch_forward_generic(p, obs, batch, out, actions, dbg_layer, dbg_acc, (int8_t *)dbg_act, st);
+}
+
+int actorq_cast_params_fp16(const actorq_layer_desc *layers, int n_layers, int head, int obs_dtype, void *cuda_stream,
+                            actorq_policy **inout_policy) {
+  if (!layers || !inout_policy) return ACTORQ_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > ACTORQ_MAX_LAYERS) return ACTORQ_ERR_INVALID_ARG;
+  if (head < ACTORQ_HEAD_TANH || head > ACTORQ_HEAD_LINEAR) return ACTORQ_ERR_INVALID_ARG;
+  if (obs_dtype != ACTORQ_OBS_F32 && obs_dtype != ACTORQ_OBS_U8_DIV255) return ACTORQ_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l].weight) return ACTORQ_ERR_INVALID_ARG;
+  actorq_policy *p = *inout_policy;
+  if (p == nullptr) {
+    p = new (std::nothrow) actorq_policy;
+    if (!p) return ACTORQ_ERR_NOMEM;
+    memset(p, 0, sizeof(*p));
+    p->n_layers = n_layers; p->head = head; p->obs_dtype = obs_dtype; p->precision = 16;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&p->device) != cudaSuccess || cudaGetDeviceProperties(&prop, p->device) != cudaSuccess) { delete p; return ACTORQ_ERR_CUDA; }
+    p->sm_count = prop.multiProcessorCount;
+    for (int l = 0; l < n_layers; ++l) {
+      int rc = fill_geometry(layers[l], p->layers[l].g);
+      if (rc == ACTORQ_OK && l > 0 && p->layers[l].g.in_elems != p->layers[l - 1].g.out_elems) rc = ACTORQ_ERR_INVALID_ARG;
+      if (rc != ACTORQ_OK) { delete p; return rc; }
+    }
+    if (!fp16_supported(p)) { delete p; return ACTORQ_ERR_UNSUPPORTED; }
+    const int rc = fp16_setup(p);
+    if (rc != ACTORQ_OK) { actorq_free(p); return rc; }
+  } else {
+    if (p->precision != 16 || p->n_layers != n_layers || p->head != head || p->obs_dtype != obs_dtype) return ACTORQ_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+      LayerGeom g;
+      const int rc = fill_geometry(layers[l], g);
+      if (rc != ACTORQ_OK) return rc;
+      if (!same_geometry(g, p->layers[l].g)) return ACTORQ_ERR_INVALID_ARG;
+    }
+  }
+  for (int l = 0; l < n_layers; ++l) { p->layers[l].w_f32 = layers[l].weight; p->layers[l].b_f32 = layers[l].bias; }
+  const int rc = launch_cast_fp16(p, (cudaStream_t)cuda_stream);
+  for (int l = 0; l < n_layers; ++l) { p->layers[l].w_f32 = nullptr; p->layers[l].b_f32 = nullptr; }
+  if (rc != ACTORQ_OK) {
+    if (*inout_policy == nullptr) actorq_free(p);
+    return rc;
+  }
+  *inout_policy = p;
+  return ACTORQ_OK;
 }
 
 int actorq_policy_forward(actorq_policy *policy, const void *obs, long long batch, float *out, int *actions,
@@ -401,6 +451,8 @@ void actorq_free(actorq_policy *p) {
   if (p->hs_mem) cudaFree(p->hs_mem);
   if (p->scratch[0]) cudaFree(p->scratch[0]);
   if (p->fcp_mem) cudaFree(p->fcp_mem);
+  if (p->f16_act) cudaFree(p->f16_act);
+  if (p->f16_pool) cudaFree(p->f16_pool);
   if (p->pool) cudaFree(p->pool);
   cudaGetLastError();
   delete p;
@@ -408,6 +460,7 @@ void actorq_free(actorq_policy *p) {
 
 int actorq_policy_export_layer_channels(actorq_policy *p, int layer, signed char *w_q, float *scales, int *zero_points,
                                         void *cuda_stream) {
+  if (p && p->precision == 16) return ACTORQ_ERR_UNSUPPORTED;      // int8 policies only
   if (!p || layer < 0 || layer >= p->n_layers || !w_q || !scales || !zero_points) return ACTORQ_ERR_INVALID_ARG;
   const LayerDev &L = p->layers[layer];
   if (!L.g.per_channel) return ACTORQ_ERR_INVALID_ARG;
@@ -421,6 +474,7 @@ int actorq_policy_export_layer_channels(actorq_policy *p, int layer, signed char
 
 int actorq_policy_export_layer(actorq_policy *p, int layer, signed char *w_q, float *scale, int *zero_point,
                                void *cuda_stream) {
+  if (p && p->precision == 16) return ACTORQ_ERR_UNSUPPORTED;      // int8 policies only
   if (!p || layer < 0 || layer >= p->n_layers || !w_q || !scale || !zero_point) return ACTORQ_ERR_INVALID_ARG;
   if (p->layers[layer].g.per_channel) return ACTORQ_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -455,24 +509,28 @@ int actorq_policy_timeout_info(actorq_policy *p, int *info8) {
 }
 
 int actorq_policy_blob_bytes(const actorq_policy *p, long long *bytes) {
+  if (p && p->precision == 16) return ACTORQ_ERR_UNSUPPORTED;
   if (!p || !bytes) return ACTORQ_ERR_INVALID_ARG;
   *bytes = blob_bytes(p);
   return ACTORQ_OK;
 }
 
 int actorq_policy_export_blob(actorq_policy *p, void *blob, long long capacity, void *cuda_stream) {
+  if (p && p->precision == 16) return ACTORQ_ERR_UNSUPPORTED;      // int8 policies only
   if (!p || !blob) return ACTORQ_ERR_INVALID_ARG;
   if (capacity < blob_bytes(p) || (reinterpret_cast<uintptr_t>(blob) & 15) != 0) return ACTORQ_ERR_INVALID_ARG;
   return launch_export_blob(p, blob, (cudaStream_t)cuda_stream);
 }
 
 int actorq_policy_import_blob(actorq_policy *p, const void *blob, long long bytes, void *cuda_stream) {
+  if (p && p->precision == 16) return ACTORQ_ERR_UNSUPPORTED;      // int8 policies only
   if (!p || !blob) return ACTORQ_ERR_INVALID_ARG;
   if (bytes != blob_bytes(p) || (reinterpret_cast<uintptr_t>(blob) & 15) != 0) return ACTORQ_ERR_INVALID_ARG;
   return launch_import_blob(p, blob, (cudaStream_t)cuda_stream);
 }
 
 int actorq_policy_set_fused_variant(actorq_policy *p, int variant) {
+  if (p && p->precision == 16) return ACTORQ_ERR_UNSUPPORTED;      // int8 policies only
   if (!p || variant < 0 || variant > 4) return ACTORQ_ERR_INVALID_ARG;
   if (variant == 3) {
     if (!p->fcp_ok) return ACTORQ_ERR_UNSUPPORTED;

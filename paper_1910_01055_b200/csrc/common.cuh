@@ -104,6 +104,15 @@ struct actorq_policy {
   int ex_seeded;
   unsigned long long ex_seed;
   long long ex_row0;
+  // the fp16 actor (fp16_pair.cu): precision 16 = the policy was cast to binary16 (actorq_cast_params_fp16),
+  // otherwise quantized to int8.  Its own pool (status block, binary16 weight images, binary32 biases) and
+  // two activation buffers grown on demand.
+  int precision;
+  void *f16_pool;
+  uint8_t *f16_img[ACTORQ_MAX_LAYERS];
+  float *f16_bias[ACTORQ_MAX_LAYERS];
+  void *f16_act;
+  long long f16_rows;
 };
 
 namespace actorq {
@@ -145,6 +154,12 @@ int launch_conv_staged(actorq_policy *p, int l, const void *in, long long batch,
                        int *dbg_acc, int8_t *dbg_act, cudaStream_t st);
 int fc_tail_run(actorq_policy *p, int l_begin, long long batch, float *out, int *actions,
                 int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st);
+
+// the fp16 actor (fp16_pair.cu)
+bool fp16_supported(const actorq_policy *p);
+int fp16_setup(actorq_policy *p);
+int launch_cast_fp16(actorq_policy *p, cudaStream_t st);
+int launch_forward_fp16(actorq_policy *p, const void *obs, long long batch, float *out, int *actions, cudaStream_t st);
 
 // out[b][n] = clamp(out[b][n] + sigma[b] * noise[b][n], -1, 1) for the paths whose head does not do it
 int launch_explore(float *out, const float *sigma, const float *noise, long long batch, int out_dim, int sm_count, cudaStream_t st);

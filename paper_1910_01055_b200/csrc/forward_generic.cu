@@ -236,6 +236,7 @@ static int static_scratch_address(int device, unsigned char **out) {
 
 extern "C" int actorq_policy_forward_noalloc(actorq_policy *p, const void *obs, long long batch, float *out,
                                              int *actions, void *cuda_stream) {
+  if (p && p->precision == 16) return ACTORQ_ERR_UNSUPPORTED;      // int8 policies only
   using namespace actorq;
   if (!p || batch < 0) return ACTORQ_ERR_INVALID_ARG;
   p->launches = 0;
