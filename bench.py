@@ -360,6 +360,8 @@ def main():
     ap.add_argument("--repeats", type=int, default=0,
                     help="how many times the K-step region is timed (default: 5 up to 500 steps, 3 up to 1000, else 1); the median repeat is reported")
     ap.add_argument("--no-int8-peak", action="store_true", help="skip the in-process measurement of the INT8 tensor peak")
+    ap.add_argument("--precision", default="int8", choices=["int8", "fp16"],
+                    help="int8: the quantized policy (the metric's path); fp16: the policy cast to binary16 (the paper's q = 16 actor), all-FC workloads")
     ap.add_argument("--ref-rows", type=int, default=2048)
     ap.add_argument("--cpu-rows", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -396,7 +398,7 @@ def main():
     batch = args.batch or cfg.get("batch") or cfg["batches"][-2]
     spec = W.build_config(args.workload)
     layers_dev = B.layers_to_device(spec)
-    pol = B.QuantizedPolicy(spec.head, spec.obs_dtype).quantize(layers_dev, spec.input_ranges)
+    pol = (B.Fp16Policy if args.precision == "fp16" else B.QuantizedPolicy)(spec.head, spec.obs_dtype).quantize(layers_dev, spec.input_ranges)
 
     # rows are sharded over ranks (weak scaling: `batch` rows per GPU per step); no collective
     # on the data path.  Inputs rotate over enough distinct batches to exceed the 126 MB L2.
@@ -515,7 +517,11 @@ def main():
         # denominator: the INT8 tensor rate measured in this process by the library's bare MMA loop
         # (burst: this bench times short regions); 2 x the measured bf16 figure only if that is skipped
         int8_peak = None
-        if not args.no_int8_peak:
+        if args.precision == "fp16":
+            peak, peak_source = float(peaks["bf16_tflops"]), f"16-bit tensor burst of {peaks['_source']} (torch bf16 matmul, {peaks['bf16_tflops']} TFLOP/s)"
+            kernel_name = "fp16_pair_kernel x layers (forward)"
+            traffic, traffic_note = None, "no ncu capture for this path"
+        elif not args.no_int8_peak:
             peak_sampler = ClockSampler(local)
             peak_sampler.start()
             int8_peak = measure_int8_peak(torch, B, pol)
@@ -524,14 +530,15 @@ def main():
                 int8_peak["clocks"] = peak_clocks
         if int8_peak is not None:
             peak, peak_source = int8_peak["burst"], "measured int8 (bare tcgen05.mma kind::i8 loop, burst, this run)"
-        else:
+        elif args.precision == "int8":
             peak_source = f"2 x bf16 burst of {peaks['_source']} ({peaks['bf16_tflops']} TFLOP/s)"
         result = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-            "config": {"workload": args.workload, "rows_per_gpu_per_step": batch,
-                       "step": "re-quantize fp32 policy to int8 + one int8 forward",
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8" if args.precision == "int8" else "f16", "data": "synthetic",
+            "config": {"workload": args.workload, "rows_per_gpu_per_step": batch, "precision": args.precision,
+                       "step": ("re-quantize fp32 policy to int8 + one int8 forward" if args.precision == "int8"
+                                else "cast fp32 policy to binary16 + one fp16 forward (not the int8 metric: the q = 16 variant)"),
                        "l2": (f"inputs rotate over {n_rot} distinct batches "
                               f"({n_rot * obs_bytes / 1e6:.0f} MB > 126 MB L2)" if flush is None
                               else "256 MB flush buffer written between timed steps"),
@@ -561,7 +568,7 @@ def main():
         if args.sweep:
             result["config"]["sweep"] = batch_sweep(torch, B, spec, pol, layers_dev,
                                                     W.CONFIGS["actor_sweep"]["batches"] if spec.obs_dtype == "f32" else [1, 16, 256, 1024])
-        if not args.no_cpu_baseline:
+        if not args.no_cpu_baseline and args.precision == "int8":
             result["cpu_baseline"], _ = cpu_baseline(spec, min(args.cpu_rows, batch))
             result["cpu_baseline"]["single_thread"] = cpu_baseline_single_thread(args.workload, min(512, args.cpu_rows, batch))
             result["int8_vs_fp"] = int8_vs_fp(torch, pol, spec, min(512, batch))

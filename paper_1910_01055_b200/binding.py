@@ -370,6 +370,15 @@ class QuantizedPolicy:
             pass
 
 
+class Fp16Policy(QuantizedPolicy):
+    """The same owner for a policy cast to binary16 (actorq_cast_params_fp16): quantize() casts."""
+
+    def quantize(self, layers: Sequence[dict], input_ranges=None, stream=None) -> "Fp16Policy":
+        self.handle = actorq_cast_params_fp16(layers, self.head, self.obs_dtype, self.handle, stream)
+        self.out_dim = layers[-1]["weight"].shape[0]
+        return self
+
+
 def layers_to_device(policy_spec, device="cuda") -> List[dict]:
     """PolicySpec (workloads.py) -> list of layer dicts holding cuda tensors."""
     out = []
