@@ -396,6 +396,11 @@ def main():
 
     cfg = W.CONFIGS[args.workload]
     batch = args.batch or cfg.get("batch") or cfg["batches"][-2]
+    # rows are independent actors: the job's batch * world rows are partitioned over the ranks in contiguous
+    # ranges (weak scaling: `batch` rows each), weights replicated, no collective on the data path
+    from paper_1910_01055_b200 import dist as D
+    first_row, end_row = D.shard_rows(batch * world, rank, world)
+    assert end_row - first_row == batch
     spec = W.build_config(args.workload)
     layers_dev = B.layers_to_device(spec)
     pol = (B.Fp16Policy if args.precision == "fp16" else B.QuantizedPolicy)(spec.head, spec.obs_dtype).quantize(layers_dev, spec.input_ranges)

@@ -176,7 +176,10 @@ int actorq_policy_forward(actorq_policy *policy, const void *obs, long long batc
  *     nothing is launched.  (DQN 4x84x84 network: 28224 elements -> batch <= 1188.)
  *   - the policy must have been quantized on the device that is current at the call.
  *   - The first call on each device looks up the array's device address (a one-time set-up that
- *     is not stream work), so make that first call before starting any stream capture.
+ *     is not stream work).  With CUDA's lazy module loading that first call is also the one that
+ *     makes the driver load the module holding the array, i.e. reserve the 64 MiB, which can
+ *     synchronise the device or fail if the memory is gone by then: make it once at start-up,
+ *     before the learner has claimed the device and before starting any stream capture.
  *   - All calls, on every policy and stream, share the one array, which simply keeps whatever the
  *     previous call left in it (nothing needs to be cleared: each call overwrites all it reads).
  *     Two calls whose kernels can overlap on the GPU therefore race; order them on one stream or

@@ -357,13 +357,24 @@ static long long host_chunk_rows(const actorq_policy *p, long long batch) {
 
 static int ensure_host_staging(actorq_policy *p, long long rows) {
   if (!p->hs_ready) {
-    if (cudaStreamCreateWithFlags(&p->hs_in, cudaStreamNonBlocking) != cudaSuccess) return ACTORQ_ERR_CUDA;
-    if (cudaStreamCreateWithFlags(&p->hs_outs, cudaStreamNonBlocking) != cudaSuccess) return ACTORQ_ERR_CUDA;
+    // all or nothing: whatever was created before a failure is destroyed again (the next call starts over)
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev[3 * actorq_policy::kHostSlots];
+    int n_ev = 0;
+    bool ok = cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess;
+    for (; ok && n_ev < 3 * actorq_policy::kHostSlots; ++n_ev)
+      if (cudaEventCreateWithFlags(&ev[n_ev], cudaEventDisableTiming) != cudaSuccess) { ok = false; break; }
+    if (!ok) {
+      for (int i = 0; i < n_ev; ++i) cudaEventDestroy(ev[i]);
+      if (s_out) cudaStreamDestroy(s_out);
+      if (s_in) cudaStreamDestroy(s_in);
+      cudaGetLastError();
+      return ACTORQ_ERR_CUDA;
+    }
+    p->hs_in = s_in; p->hs_outs = s_out;
     for (int i = 0; i < actorq_policy::kHostSlots; ++i) {
-      if (cudaEventCreateWithFlags(&p->hs_ev_in[i], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&p->hs_ev_comp[i], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&p->hs_ev_out[i], cudaEventDisableTiming) != cudaSuccess)
-        return ACTORQ_ERR_CUDA;
+      p->hs_ev_in[i] = ev[3 * i]; p->hs_ev_comp[i] = ev[3 * i + 1]; p->hs_ev_out[i] = ev[3 * i + 2];
     }
     p->hs_ready = 1;
   }

@@ -419,53 +419,14 @@ conv_gemm_kernel(const __grid_constant__ ConvGemmArgs A) {
   }
 }
 
-// Input quantizer for the all-FC form (Eq. 1 on the observations, one binary32 multiply by 1 / s_a):
-// float rows [batch][K] -> int8 rows of `stride` bytes (the padding bytes are never used: the gather
-// masks K positions beyond the layer's reduction length).
-__global__ void quantize_obs_rows_kernel(const float *__restrict__ x, long long batch, int K, int stride,
-                                         const LayerParams *__restrict__ params, int8_t *__restrict__ q) {
-  const LayerParams p = params[0];
-  const float lo_f = (float)(-128 - p.z_a), hi_f = (float)(127 - p.z_a);
-  const long long total = batch * stride;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-    const long long b = i / stride;
-    const int k = (int)(i - b * stride);
-    int code = 0;
-    if (k < K) {
-      float t = __fmul_rn(__ldg(x + b * K + k), p.inv_s_a);
-      if (t != t) t = 0.0f;                                    // NaN -> real 0
-      t = fminf(fmaxf(t, lo_f), hi_f);
-      code = __float2int_rn(t) + p.z_a;
-    }
-    q[i] = (int8_t)code;
-  }
-}
-
 // ---- host side ------------------------------------------------------------------------------
 
 static int cg_round_up(int v, int m) { return (v + m - 1) / m * m; }
 
-// Which input layout layer l reads on this path, or -1 if the policy cannot take the path.
-//   layer 0: uint8 NCHW frames into a convolution whose rows can be read 4 bytes at a time
-//   later layers: int8 NHWC with a multiple of 16 channels (an FC layer counts its whole input
-//   as channels when it follows an FC layer, and as (c, h, w) -> (h, w, c) when it follows a conv)
-// All-FC policies on float observations that the fused MLP kernels do not take (layers wider than
-// 1024, e.g. the paper's 2048-wide ActorQ policies) also run here, one launch per layer: a small
-// kernel quantizes the observations to int8 rows (padded to 16 bytes), and every layer is then the
-// "FC after FC" case of this kernel.
-static bool fc_gemm_supported(const actorq_policy *p) {
-  if (p->obs_dtype != ACTORQ_OBS_F32 || p->n_layers < 2) return false;
-  for (int l = 0; l < p->n_layers; ++l) {
-    const LayerGeom &g = p->layers[l].g;
-    const bool last = (l + 1 == p->n_layers);
-    if (g.kind != ACTORQ_FC) return false;
-    if (last ? g.N > 128 : (g.N > 4096 || (g.N & 15))) return false;
-  }
-  return true;
-}
-
+// Policies this path takes: uint8 NCHW frames into a convolution whose rows can be read 4 bytes at a
+// time; later layers read int8 NHWC with a multiple of 16 channels (an FC layer counts (c, h, w) ->
+// (h, w, c) when it follows a convolution, its whole input as channels when it follows an FC layer).
 bool conv_gemm_supported(const actorq_policy *p) {
-  if (fc_gemm_supported(p)) return true;
   if (p->obs_dtype != ACTORQ_OBS_U8_DIV255 || p->n_layers < 2) return false;
   const LayerGeom &g0 = p->layers[0].g;
   if (g0.kind != ACTORQ_CONV2D) return false;
@@ -530,16 +491,6 @@ int launch_forward_conv_gemm(actorq_policy *p, const void *obs, long long batch,
   }
   const void *cur = obs;
   int8_t *bufs[2] = {p->scratch[0], p->scratch[1]};
-  const bool f32_obs = (p->obs_dtype == ACTORQ_OBS_F32);
-  const int k0_stride = cg_round_up(p->layers[0].g.K, 16);
-  if (f32_obs) {          // observation rows -> int8 codes, rows 16-byte aligned; layer 0 writes bufs[0]
-    const long long total = batch * k0_stride;
-    long long blocks = (total + 255) / 256;
-    if (blocks > (long long)p->sm_count * 32) blocks = (long long)p->sm_count * 32;
-    quantize_obs_rows_kernel<<<(int)blocks, 256, 0, st>>>((const float *)obs, batch, p->layers[0].g.K, k0_stride, p->d_params, bufs[1]);
-    p->launches++;
-    cur = bufs[1];
-  }
   // The fully connected layers behind the last convolution run on the CTA-pair layer kernel
   // (fc_pair.cu), fed directly by that convolution's epilogue; where it cannot take them (or no
   // pair of CTAs can be scheduled) they run here like every other layer.
@@ -550,7 +501,7 @@ int launch_forward_conv_gemm(actorq_policy *p, const void *obs, long long batch,
   int *rs_all = nullptr;          // the tail's row-sum counters: cleared by the kernel of layer l_tail - 2 when that is a
   long long rs_all_len = 0;       // staged convolution (no memset between the kernels of consecutive forwards)
   bool clear_in_kernel = false;
-  if (!f32_obs) {
+  {
     int lc = -1;
     for (int l = 0; l < p->n_layers; ++l)
       if (p->layers[l].g.kind == ACTORQ_CONV2D) lc = l;
@@ -563,7 +514,7 @@ int launch_forward_conv_gemm(actorq_policy *p, const void *obs, long long batch,
     const LayerDev &L = p->layers[l];
     const LayerGeom &g = L.g;
     const bool last = (l + 1 == p->n_layers);
-    if (!f32_obs && conv_staged_supported(p, l, batch)) {      // convolutions: input staged in shared memory
+    if (conv_staged_supported(p, l, batch)) {      // convolutions: input staged in shared memory
       const bool feeds_tail = (l + 1 == l_tail && l_tail < p->n_layers);
       const bool clears = clear_in_kernel && l_tail < p->n_layers && l == l_tail - 2;
       const int rc = launch_conv_staged(p, l, cur, batch, feeds_tail ? nullptr : bufs[l & 1], feeds_tail ? blk : nullptr,
@@ -576,14 +527,14 @@ int launch_forward_conv_gemm(actorq_policy *p, const void *obs, long long batch,
     }
     ConvGemmArgs A;
     memset(&A, 0, sizeof(A));
-    A.in_mode = (l == 0 && !f32_obs) ? 0 : 1;
+    A.in_mode = (l == 0) ? 0 : 1;
     if (g.kind == ACTORQ_CONV2D) {
       A.C = g.in_c; A.H = g.in_h; A.W = g.in_w; A.stride = g.stride; A.OH = g.out_h; A.OW = g.out_w;
     } else if (l > 0 && p->layers[l - 1].g.kind == ACTORQ_CONV2D) {
       const LayerGeom &gp = p->layers[l - 1].g;
       A.C = gp.out_c; A.H = gp.out_h; A.W = gp.out_w; A.stride = 1; A.OH = 1; A.OW = 1;
     } else {
-      A.C = (l == 0) ? k0_stride : g.K; A.H = 1; A.W = 1; A.stride = 1; A.OH = 1; A.OW = 1;   // C: bytes between rows
+      A.C = g.K; A.H = 1; A.W = 1; A.stride = 1; A.OH = 1; A.OW = 1;   // C: bytes between rows
     }
     A.K = g.K; A.Kpad = cg_round_up(g.K, 32); A.nkb = (g.K + 127) / 128;
     A.N = g.N; A.Npad = cg_round_up(g.N, 16); A.nchunk = (A.Npad + kChunkN - 1) / kChunkN;

@@ -163,10 +163,11 @@ int launch_explore(float *out, const float *sigma, const float *noise, long long
   return cuda_ok(cudaGetLastError());
 }
 
-int launch_forward_generic(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
-                           int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st) {
+// The layer-at-a-time forward with its two int8 activation buffers given by the caller: the policy's
+// scratch (launch_forward_generic) or the fixed array of the allocation-free entry point.
+static int run_generic_layers(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
+                              int dbg_layer, int *dbg_acc, int8_t *dbg_act, int8_t *cur, int8_t *nxt, cudaStream_t st) {
   const int sm = p->sm_count;
-  int8_t *cur = p->scratch[0], *nxt = p->scratch[1];
   const long long n0 = batch * p->layers[0].g.in_elems;
   if (p->obs_dtype == ACTORQ_OBS_U8_DIV255)
     quantize_obs_u8_kernel<<<grid_for(n0, 256, sm), 256, 0, st>>>((const uint8_t *)obs, n0, cur);
@@ -204,6 +205,11 @@ int launch_forward_generic(actorq_policy *p, const void *obs, long long batch, f
     p->launches++;
   }
   return cuda_ok(cudaGetLastError());
+}
+
+int launch_forward_generic(actorq_policy *p, const void *obs, long long batch, float *out, int *actions,
+                           int dbg_layer, int *dbg_acc, int8_t *dbg_act, cudaStream_t st) {
+  return run_generic_layers(p, obs, batch, out, actions, dbg_layer, dbg_acc, dbg_act, p->scratch[0], p->scratch[1], st);
 }
 
 // ---- forward without any allocation -----------------------------------------------------------
@@ -264,43 +270,5 @@ extern "C" int actorq_policy_forward_noalloc(actorq_policy *p, const void *obs, 
 
   // Nothing in the array has to start at zero: the input quantizer writes every element the first
   // layer reads, and each layer writes every element the next one reads.
-  cudaStream_t st = (cudaStream_t)cuda_stream;
-  const int sm = p->sm_count;
-  const long long n0 = batch * p->layers[0].g.in_elems;
-  if (p->obs_dtype == ACTORQ_OBS_U8_DIV255)
-    quantize_obs_u8_kernel<<<grid_for(n0, 256, sm), 256, 0, st>>>((const uint8_t *)obs, n0, cur);
-  else
-    quantize_obs_f32_kernel<<<grid_for(n0, 256, sm), 256, 0, st>>>((const float *)obs, n0, p->d_params, cur);
-  p->launches++;
-  for (int l = 0; l < p->n_layers; ++l) {
-    const LayerDev &L = p->layers[l];
-    const bool last = (l + 1 == p->n_layers);
-    GenericLayerArgs A;
-    A.g = L.g;
-    A.a = cur;
-    A.wq = L.wq;
-    A.bias_q = L.bias_q;
-    A.ch_zw = L.g.per_channel ? L.ch_zw : nullptr;
-    A.ch_M = L.g.per_channel ? L.ch_M : nullptr;
-    A.ch_P = L.g.per_channel ? L.ch_P : nullptr;
-    A.a_next = last ? nullptr : nxt;
-    A.y = last ? out : nullptr;
-    A.dbg_acc = nullptr;
-    A.dbg_act = nullptr;
-    A.apply_tanh = (p->head == ACTORQ_HEAD_TANH);
-    A.layer = l;
-    A.batch = batch;
-    const long long work = batch * L.g.out_elems;
-    if (L.g.kind == ACTORQ_CONV2D)
-      conv_generic_kernel<<<grid_for(work, 256, sm), 256, 0, st>>>(A, p->d_params);
-    else
-      fc_generic_kernel<<<grid_for(work, 256, sm), 256, 0, st>>>(A, p->d_params);
-    p->launches++;
-    int8_t *t = cur; cur = nxt; nxt = t;
-  }
-  if (p->head == ACTORQ_HEAD_ARGMAX) {
-    argmax_kernel<<<grid_for(batch, 128, sm), 128, 0, st>>>(out, batch, p->layers[p->n_layers - 1].g.N, actions);
-    p->launches++;
-  }
-  return cuda_ok(cudaGetLastError());
+  return run_generic_layers(p, obs, batch, out, actions, -1, nullptr, nullptr, cur, nxt, (cudaStream_t)cuda_stream);
 }
