@@ -22,19 +22,21 @@
 // sum of its codes, exactly.  The layer's whole weight image stays resident in shared memory (its
 // column constants too); tensor memory holds two accumulators, so gather, MMAs and epilogue of
 // neighbouring tiles overlap.
-// Warps: 0 bulk-copy producer, 1 MMA issuer, 2-17 gather, 18-21 epilogue (TMEM lane quarters).
+// Warps: 0 bulk-copy producer, 1 MMA issuer, 2-9 gather, 10-17 epilogue (two sets of four, one per
+// accumulator; a warp per TMEM lane quarter).
 // Every wait is bounded (ACTORQ_ERR_TIMEOUT in the status word, all roles leave, TMEM is freed).
 #include "tcgen05.cuh"
 
 namespace actorq {
 namespace cst {
 
-constexpr int kThreads = 704;
+constexpr int kThreads = 576;
 constexpr int kGatherWarp0 = 2;
-constexpr int kGatherWarps = 16;
-constexpr int kRowsInFlight = kTileM / kGatherWarps;    // a warp's rows of a tile, all in flight at once
-constexpr int kEpiWarp0 = 18;
-constexpr int kEpiWarps = 4;
+constexpr int kGatherWarps = 8;        // (a multiple of 8: a warp's rows, kGatherWarps apart, share row & 7, the swizzle phase)
+constexpr int kRowsWarp = kTileM / kGatherWarps;        // a warp's rows of a tile, gathered kRowsInFlight at a time
+constexpr int kRowsInFlight = 8;
+constexpr int kEpiWarp0 = 10;
+constexpr int kEpiWarps = 8;           // two sets of four (one warp per TMEM lane quarter); set s takes the tiles in accumulator s
 constexpr int kMaxStages = 8;
 constexpr int kAccBufs = 2;            // accumulators in tensor memory (acc_stride columns each)
 
@@ -85,6 +87,60 @@ struct __align__(16) Barriers {
   int abort_flag;
 };
 
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t lo, uint32_t hi) {
+  asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(lo), "r"(hi) : "memory");
+}
+
+// kRowsInFlight operand rows of a tile, one warp instruction per row and step; nothing in the loop depends
+// on the row.  Rows past the item's last one read whatever the staging buffer holds: their accumulators
+// are never used (operand rows are independent of one another).
+//   rs       the rows' entries of the row-offset table (kGatherWarps apart)
+//   src[st]  shared address of the staged input + the lane's offset inside a receptive field
+//   dst[st]  shared address of the lane's bytes in the first of the rows (swizzle folded in); rows kGatherWarps * 128 apart
+// kPlanes: uint8 NCHW input, 8 bytes per lane (code = u - 128), else int8 NHWC, 16 bytes per lane.
+template <bool kPlanes>
+__device__ __forceinline__ void gather_rows(const int *rs, const uint32_t (&src)[2], const uint32_t (&dst)[2],
+                                            const bool (&data_ok)[2], const bool (&slot_ok)[2]) {
+  constexpr int U = kRowsInFlight;
+  constexpr uint32_t kDstStride = (uint32_t)kGatherWarps << 7;
+  uint32_t off[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) off[u] = (uint32_t)rs[u * kGatherWarps];
+#pragma unroll
+  for (int st = 0; st < 2; ++st) {
+    if (!slot_ok[st]) continue;
+    if (kPlanes) {
+      uint32_t lo[U], hi[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        lo[u] = 0u; hi[u] = 0u;
+        if (data_ok[st]) { lo[u] = lds32(src[st] + off[u]) ^ 0x80808080u; hi[u] = lds32(src[st] + off[u] + 4) ^ 0x80808080u; }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) sts64(dst[st] + (uint32_t)u * kDstStride, lo[u], hi[u]);
+    } else {
+      uint4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) v[u] = data_ok[st] ? lds128(src[st] + off[u]) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int u = 0; u < U; ++u) sts128(dst[st] + (uint32_t)u * kDstStride, v[u]);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 conv_staged_kernel(const __grid_constant__ Args A) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -109,7 +165,7 @@ conv_staged_kernel(const __grid_constant__ Args A) {
     mbar_init(&bars->w_ready, kEpiWarps);
     for (int b = 0; b < 2; ++b) { mbar_init(&bars->in_full[b], 1); mbar_init(&bars->in_empty[b], kGatherWarps); }
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(&bars->a_full[s], kGatherWarps); mbar_init(&bars->a_empty[s], 1); }
-    for (int b = 0; b < kAccBufs; ++b) { mbar_init(&bars->acc_full[b], 1); mbar_init(&bars->acc_empty[b], kEpiWarps); }
+    for (int b = 0; b < kAccBufs; ++b) { mbar_init(&bars->acc_full[b], 1); mbar_init(&bars->acc_empty[b], 4); }
     mbar_init(&bars->drain, 1);
     bars->abort_flag = 0;
     if (blockIdx.x == 0) A.status[7] = (int)smem_u32(bars);
@@ -226,14 +282,15 @@ conv_staged_kernel(const __grid_constant__ Args A) {
     volatile int never = 0;
     mbar_wait_warp(&bars->drain, 0, &never, A.status);
   } else if (warp < kEpiWarp0) {
-    // ---------------- gather (warps 2..17): a warp per output pixel, lanes over the receptive field ----------------
+    // ---------------- gather (warps 2..9): a warp per output pixel, lanes over the receptive field ----------------
     const int gw = warp - kGatherWarp0;
     // what this lane fetches in each of the (at most two) steps over a row's K bytes:
     //   mode 1: 16-byte piece j = 32 step + lane of the row, K order (kh, kw, c): input offset of its 16 channels
     //   mode 0: 8 bytes q = 32 step + lane = (c, kh): input row segment kw = 0..7 (lane pairs form a 16-byte piece)
     int src_off[2], piece[2];
+    uint32_t dst_lane[2];     // the lane's bytes in row gw of a ring stage; its rows, kGatherWarps apart, share row & 7
     bool data_ok[2], slot_ok[2];
-    const int n_steps = (A.in_mode == 1) ? ((A.Kpad >> 4) + 31) >> 5 : ((A.Kpad >> 3) + 31) >> 5;
+    const uint32_t ring_addr = smem_u32(a_ring);
 #pragma unroll
     for (int st = 0; st < 2; ++st) {
       const int j = st * 32 + lane;
@@ -244,12 +301,14 @@ conv_staged_kernel(const __grid_constant__ Args A) {
         piece[st] = j;
         data_ok[st] = j < (A.K >> 4);
         slot_ok[st] = j < (A.Kpad >> 4);
+        dst_lane[st] = ((uint32_t)gw << 7) + (((uint32_t)(piece[st] ^ gw) & 7) << 4);
       } else {
         const int c = j / A.KH, kh = j - c * A.KH;
         src_off[st] = c * A.plane_pitch + kh * A.W;
         piece[st] = j >> 1;
         data_ok[st] = j < A.C * A.KH;
         slot_ok[st] = j < (A.Kpad >> 3);                    // every lane stores its 8 bytes (half of a 16-byte piece)
+        dst_lane[st] = ((uint32_t)gw << 7) + (((uint32_t)(piece[st] ^ gw) & 7) << 4) + ((uint32_t)(lane & 1) << 3);
       }
     }
     int s = 0;
@@ -257,14 +316,14 @@ conv_staged_kernel(const __grid_constant__ Args A) {
     bool ok = true;
     for (long long item = blockIdx.x; item < A.n_items && ok; item += gridDim.x, ++i) {
       const int buf = i & 1;
-      const int rows_valid = item_samples(item) * ohw;
-      const int n_tiles = (rows_valid + kTileM - 1) / kTileM;
+      const int n_tiles = (item_samples(item) * ohw + kTileM - 1) / kTileM;
       ok = mbar_wait_warp(&bars->in_full[buf], (i >> 1) & 1, abort_flag, A.status);
       if (!ok) break;
-      const uint8_t *in_buf = in_s + buf * in_bytes;
+      const uint32_t in_addr = smem_u32(in_s + buf * in_bytes);
+      const uint32_t src[2] = {in_addr + (uint32_t)src_off[0], in_addr + (uint32_t)src_off[1]};
       for (int t = 0; t < n_tiles && ok; ++t, ++tc) {
         // the tile's nkb operand stages: wait until the MMAs that read their previous contents are done
-        uint32_t stage_base[2];
+        uint32_t stage_base[2] = {0u, 0u};
         {
           int s2 = s;
           uint32_t ph2 = ph;
@@ -273,63 +332,20 @@ conv_staged_kernel(const __grid_constant__ Args A) {
             if (!ok) break;
 #pragma unroll
             for (int st = 0; st < 2; ++st)
-              if ((piece[st] >> 3) == kb) stage_base[st] = (uint32_t)s2 * kStageBytes + (((uint32_t)piece[st] & 7) << 4);
+              if ((piece[st] >> 3) == kb) stage_base[st] = (uint32_t)s2 * kStageBytes;
             if (++s2 == A.n_a) { s2 = 0; ph2 ^= 1; }
           }
           if (!ok) break;
         }
-        // the warp's rows of the tile all at once, so that their loads, shuffles and stores overlap
-        // (one row alone is a chain of shared-memory latencies; the gather is bound by them, not by issue)
-        constexpr int kR = kRowsInFlight;
-        {
-          const int r0 = gw;
-          const uint8_t *src[kR];
-          bool r_ok[kR];
+        // the warp's rows, kRowsInFlight at a time so that their loads and stores overlap (one row alone is a
+        // chain of shared-memory latencies)
+        const uint32_t dst[2] = {ring_addr + stage_base[0] + dst_lane[0], ring_addr + stage_base[1] + dst_lane[1]};
 #pragma unroll
-          for (int u = 0; u < kR; ++u) {
-            const int ir = t * kTileM + r0 + u * kGatherWarps;
-            r_ok[u] = ir < rows_valid;
-            src[u] = in_buf + row_src[ir];
-          }
-          if (A.in_mode == 1) {
-#pragma unroll
-            for (int st = 0; st < 2; ++st) {
-              if (st >= n_steps) break;
-              uint4 v[kR];
-#pragma unroll
-              for (int u = 0; u < kR; ++u) {
-                v[u] = make_uint4(0u, 0u, 0u, 0u);
-                if (data_ok[st] && r_ok[u]) v[u] = *reinterpret_cast<const uint4 *>(src[u] + src_off[st]);
-              }
-#pragma unroll
-              for (int u = 0; u < kR; ++u) {
-                const int r = r0 + u * kGatherWarps;
-                if (slot_ok[st] && r_ok[u])
-                  *reinterpret_cast<uint4 *>(a_ring + ((uint32_t)r << 7) + (stage_base[st] ^ (((uint32_t)r & 7) << 4))) = v[u];
-              }
-            }
-          } else {
-#pragma unroll
-            for (int st = 0; st < 2; ++st) {
-              if (st >= n_steps) break;
-              uint32_t lo[kR], hi[kR];
-#pragma unroll
-              for (int u = 0; u < kR; ++u) {
-                lo[u] = 0u; hi[u] = 0u;
-                if (data_ok[st] && r_ok[u]) {                  // code = u - 128
-                  lo[u] = *reinterpret_cast<const uint32_t *>(src[u] + src_off[st]) ^ 0x80808080u;
-                  hi[u] = *reinterpret_cast<const uint32_t *>(src[u] + src_off[st] + 4) ^ 0x80808080u;
-                }
-              }
-#pragma unroll
-              for (int u = 0; u < kR; ++u) {
-                const int r = r0 + u * kGatherWarps;
-                if (slot_ok[st] && r_ok[u])                // the odd lane of a pair fills the upper 8 bytes of the piece
-                  *reinterpret_cast<uint2 *>(a_ring + ((uint32_t)r << 7) + (stage_base[st] ^ (((uint32_t)r & 7) << 4)) + ((lane & 1) << 3)) =
-                      make_uint2(lo[u], hi[u]);
-              }
-            }
-          }
+        for (int u0 = 0; u0 < kRowsWarp; u0 += kRowsInFlight) {
+          const int *rs = row_src + t * kTileM + gw + u0 * kGatherWarps;
+          const uint32_t d[2] = {dst[0] + ((uint32_t)(u0 * kGatherWarps) << 7), dst[1] + ((uint32_t)(u0 * kGatherWarps) << 7)};
+          if (A.in_mode == 1) gather_rows<false>(rs, src, d, data_ok, slot_ok);
+          else gather_rows<true>(rs, src, d, data_ok, slot_ok);
         }
         fence_proxy_async();
         __syncwarp();
@@ -342,8 +358,9 @@ conv_staged_kernel(const __grid_constant__ Args A) {
       if (ok && lane == 0) mbar_arrive(&bars->in_empty[buf]);     // this warp is done with the staged input
     }
   } else {
-    // ---------------- epilogue (warps 18..21): one warp per TMEM lane quarter ----------------
+    // ---------------- epilogue (warps 10..17): two sets, one warp per TMEM lane quarter each ----------------
     const int quarter = warp & 3;
+    const uint32_t set = (uint32_t)(warp - kEpiWarp0) >> 2;      // this warp's accumulator: tiles tc with tc % 2 == set
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const LayerParams p = A.params[A.layer];
@@ -367,6 +384,7 @@ conv_staged_kernel(const __grid_constant__ Args A) {
       const int n_tiles = (rows_valid + kTileM - 1) / kTileM;
       for (int t = 0; t < n_tiles && ok; ++t, ++tc) {
         const uint32_t buf = tc & (kAccBufs - 1), use = tc / kAccBufs;
+        if (buf != set) continue;
         ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_full[buf], use & 1, abort_flag, A.status));
         if (!ok) break;
         tc_fence_after();
