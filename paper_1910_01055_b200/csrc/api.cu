@@ -226,8 +226,14 @@ static int forward_impl(actorq_policy *p, const void *obs, long long batch, floa
     return launch_forward_fp16(p, obs, batch, out, actions, st);
   }
   // Wide all-FC policies (and any all-FC policy when the caller asks for it): one launch per layer
-  // on CTA pairs, activations as MMA operand blocks in device memory.
-  if ((p->fused_variant == 3 || !p->fused_ok) && p->fcp_ok) {
+  // on CTA pairs, activations as MMA operand blocks in device memory.  With a hidden layer wider than
+  // 512 the fused kernels hold one accumulator per tile (their tensor memory also carries the
+  // activations) and pause the MMAs at every hand-over; the layer kernel alternates two accumulators
+  // and spreads a layer's (row tile, column chunk) items over all CTA pairs, which wins from a few
+  // thousand rows up to the largest batches.
+  bool wide = false;
+  for (int l = 0; l + 1 < p->n_layers; ++l) wide = wide || p->layers[l].g.N > 512;
+  if ((p->fused_variant == 3 || !p->fused_ok || (p->fused_variant == 0 && wide)) && p->fcp_ok) {
     const int rc = launch_forward_fc_pair(p, obs, batch, out, actions, dbg_layer, dbg_acc, (int8_t *)dbg_act, st);
     if (rc != ACTORQ_ERR_UNSUPPORTED || p->fused_variant == 3) return rc;
     p->launches = 0;

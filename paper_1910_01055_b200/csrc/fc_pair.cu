@@ -391,7 +391,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
         // running maximum per row); warps of later parts only hand the accumulator back ----
         const bool split = (A.head != ACTORQ_HEAD_ARGMAX);
         const int n_slices = (part == 0 || (split && part == 1)) ? (rows_c + 31) / 32 : 0;
-        const int sub = split ? part * 16 : 0, jmax = split ? 4 : 8;
+        const int sub = split ? part * 16 : 0;
         float best_v = 0.0f;
         int best_n = -1;
         if (n_slices == 0) {
@@ -399,46 +399,57 @@ fc_pair_kernel(const __grid_constant__ Args A) {
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8u * buf);
         }
-        for (int s = 0; s < n_slices; ++s) {
-          const int col0 = s * 32 + sub;
+        // (every column of the slice is computed, without branches, so that the tanh chains of a thread's
+        // columns overlap; columns past N only never leave: the constant arrays are zero-padded)
+        auto head_slice = [&](auto width, int col0, bool last_slice) {
+          constexpr int kW = decltype(width)::value;          // columns per thread: 16 (split) or 32
           uint32_t r[32];
-          tmem_ld32_wait(acc + col0, r);     // (a split warp uses the first 16 of them)
-          if (s + 1 == n_slices) {
+          tmem_ld32_wait(acc + col0, r);                      // (a split warp uses the first 16 of them)
+          if (last_slice) {                                   // the accumulator goes back before the arithmetic
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8u * buf);
           }
           const int n0 = col0;
-          const int4 *cc4 = reinterpret_cast<const int4 *>(A.cc + n0);
+          int ccv[kW];
 #pragma unroll
-          for (int j4 = 0; j4 < 8; ++j4) {
-            if (j4 >= jmax) break;
-            const int4 cc = __ldg(cc4 + j4);
-            const int ccv[4] = {cc.x, cc.y, cc.z, cc.w};
+          for (int j4 = 0; j4 < kW / 4; ++j4) {
+            const int4 cc = __ldg(reinterpret_cast<const int4 *>(A.cc + n0) + j4);
+            ccv[4 * j4] = cc.x; ccv[4 * j4 + 1] = cc.y; ccv[4 * j4 + 2] = cc.z; ccv[4 * j4 + 3] = cc.w;
+          }
+          float y[kW];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int n = n0 + 4 * j4 + e;
-              if (n < A.N) {
-                const int av = (int)(r[4 * j4 + e] + (uint32_t)ccv[e] + (uint32_t)(kPC ? -__ldg(A.ch_zw + n) * rs_in : rterm));
-                if (kDbg && A.dbg_acc != nullptr && row_valid) A.dbg_acc[grow * A.N + n] = av;
-                float y = __fmul_rn(__int2float_rn(av), kPC ? __ldg(A.ch_P + n) : p.P);          // Eq. 3 on the accumulator
-                if (y > best_v || best_n < 0) { best_v = y; best_n = n; }
-                if (A.head == ACTORQ_HEAD_TANH) {
-                  y = tanhf(y);
-                  if (A.noise != nullptr && row_valid) {     // actor exploration: y + sigma * eps, kept in [-1, 1]
-                    y = __fadd_rn(y, __fmul_rn(sigma_row, __ldg(A.noise + grow * A.N + n)));
-                    y = fminf(fmaxf(y, -1.0f), 1.0f);
-                  }
+          for (int j = 0; j < kW; ++j) {
+            const int av = (int)(r[j] + (uint32_t)ccv[j] + (uint32_t)(kPC ? -__ldg(A.ch_zw + n0 + j) * rs_in : rterm));
+            if (kDbg && A.dbg_acc != nullptr && row_valid && n0 + j < A.N) A.dbg_acc[grow * A.N + n0 + j] = av;
+            y[j] = __fmul_rn(__int2float_rn(av), kPC ? __ldg(A.ch_P + n0 + j) : p.P);          // Eq. 3 on the accumulator
+          }
+          if (A.head == ACTORQ_HEAD_ARGMAX) {
+#pragma unroll
+            for (int j = 0; j < kW; ++j)
+              if (n0 + j < A.N && (y[j] > best_v || best_n < 0)) { best_v = y[j]; best_n = n0 + j; }
+          } else if (A.head == ACTORQ_HEAD_TANH) {
+#pragma unroll
+            for (int j = 0; j < kW; ++j) y[j] = tanhf(y[j]);
+            if (A.noise != nullptr && row_valid) {            // actor exploration: y + sigma * eps, kept in [-1, 1]
+#pragma unroll
+              for (int j = 0; j < kW; ++j)
+                if (n0 + j < A.N) {
+                  const float t = __fadd_rn(y[j], __fmul_rn(sigma_row, __ldg(A.noise + grow * A.N + n0 + j)));
+                  y[j] = fminf(fmaxf(t, -1.0f), 1.0f);
                 }
-                r[4 * j4 + e] = __float_as_uint(y);
-              }
             }
           }
+#pragma unroll
+          for (int j = 0; j < kW; ++j) r[j] = __float_as_uint(y[j]);
           // the warp's 32 rows x 16 (32) columns leave through shared memory, row segments coalesced
           const long long wrow0 = tile * kTileM + quarter * 32;
           const int rows_valid = (int)max(0ll, min(32ll, A.batch - wrow0));
-          if (split) warp_store_rows<16>(A.out, wrow0, rows_valid, A.N, n0, r, head_buf + ew * 512, lane);
-          else warp_store_rows<32>(A.out, wrow0, rows_valid, A.N, n0, r, head_buf + ew * 1024, lane);
+          warp_store_rows<kW>(A.out, wrow0, rows_valid, A.N, n0, r, head_buf + ew * (32 * kW), lane);
+        };
+        for (int s = 0; s < n_slices; ++s) {
+          if (split) head_slice(PathC<16>{}, s * 32 + sub, s + 1 == n_slices);
+          else head_slice(PathC<32>{}, s * 32, s + 1 == n_slices);
         }
         if (A.head == ACTORQ_HEAD_ARGMAX && part == 0 && row_valid) A.actions[grow] = best_n;
       }

@@ -287,15 +287,19 @@ fp16_pair_kernel(const __grid_constant__ Args A) {
             *reinterpret_cast<uint4 *>(rowp + (((p0 + q) ^ ((uint32_t)row & 7u)) << 4)) =
                 make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
         } else {
+          // (all 32 columns without branches, so that the tanh chains overlap; columns >= N never leave)
+          if (A.head == ACTORQ_HEAD_ARGMAX) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int n = n0 + j;
-            if (n < A.N) {
-              float y = v[j];
-              if (y > best_v || best_n < 0) { best_v = y; best_n = n; }
-              if (A.head == ACTORQ_HEAD_TANH) y = tanhf(y);
-              if (row_valid) A.out[grow * A.N + n] = y;
-            }
+            for (int j = 0; j < 32; ++j)
+              if (n0 + j < A.N && (v[j] > best_v || best_n < 0)) { best_v = v[j]; best_n = n0 + j; }
+          } else if (A.head == ACTORQ_HEAD_TANH) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = tanhf(v[j]);
+          }
+          if (row_valid) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n0 + j < A.N) A.out[grow * A.N + n0 + j] = v[j];
           }
         }
       }

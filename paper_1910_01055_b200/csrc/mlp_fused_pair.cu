@@ -472,47 +472,62 @@ fused_mlp_pair_kernel(const __grid_constant__ Args A) {
             // greedy-action head is done by the half-0 warps alone (one running maximum per row)
             const bool split = (A.head != ACTORQ_HEAD_ARGMAX);
             const int n_slices = (split || half == 0) ? (rows_c + 31) / 32 : 0;
-            const int sub = split ? half * 16 : 0, jmax = split ? 4 : 8;
+            const int sub = split ? half * 16 : 0;
             if (n_slices == 0) {
               tc_fence_before();
               __syncwarp();
               if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
             }
-            for (int s = 0; s < n_slices; ++s) {
-              const int col0 = s * 32 + sub;
+            // (every column of a slice is computed, without branches, so that the tanh chains of a thread's
+            // columns overlap; columns past N never leave: the constants in shared memory are zero-padded)
+            auto head_slice = [&](auto width, int col0, bool last_slice) {
+              constexpr int kW = decltype(width)::value;          // columns per thread: 16 (split) or 32
               uint32_t r[32];
-              tmem_ld32_wait(tmem + lane_addr + col0, r);     // (a split warp uses the first 16 of them)
-              if (s + 1 == n_slices) {
+              tmem_ld32_wait(tmem + lane_addr + col0, r);         // (a split warp uses the first 16 of them)
+              if (last_slice) {
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
               }
               const int n0 = c * kAccCols + col0;
               const int4 *cc4 = cc_buf + (n0 >> 2);
+              float y[kW];
 #pragma unroll
-              for (int j4 = 0; j4 < 8; ++j4) {
-                if (j4 >= jmax) break;
-                int4 cc = cc4[j4];
+              for (int j4 = 0; j4 < kW / 4; ++j4) {
+                const int4 cc = cc4[j4];
                 const int ccv[4] = {cc.x, cc.y, cc.z, cc.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                  const int n = n0 + 4 * j4 + e;
                   const int acc = (int)(r[4 * j4 + e] + (uint32_t)ccv[e] + (uint32_t)rterm);
-                  if (n < L.N) {
-                    if (dbg && row_valid) A.dbg_acc[grow * L.N + n] = acc;
-                    float y = __fmul_rn(__int2float_rn(acc), p.P);          // Eq. 3 on the accumulator
-                    if (y > best_v || best_n < 0) { best_v = y; best_n = n; }
-                    if (A.head == ACTORQ_HEAD_TANH) {
-                      y = tanhf(y);
-                      if (A.noise != nullptr && row_valid) {     // actor exploration: y + sigma * eps, kept in [-1, 1]
-                        y = __fadd_rn(y, __fmul_rn(sigma_row, __ldg(A.noise + grow * A.out_dim + n)));
-                        y = fminf(fmaxf(y, -1.0f), 1.0f);
-                      }
-                    }
-                    if (row_valid) A.out[grow * A.out_dim + n] = y;
-                  }
+                  if (dbg && row_valid && n0 + 4 * j4 + e < L.N) A.dbg_acc[grow * L.N + n0 + 4 * j4 + e] = acc;
+                  y[4 * j4 + e] = __fmul_rn(__int2float_rn(acc), p.P);          // Eq. 3 on the accumulator
                 }
               }
+              if (A.head == ACTORQ_HEAD_ARGMAX) {
+#pragma unroll
+                for (int j = 0; j < kW; ++j)
+                  if (n0 + j < L.N && (y[j] > best_v || best_n < 0)) { best_v = y[j]; best_n = n0 + j; }
+              } else if (A.head == ACTORQ_HEAD_TANH) {
+#pragma unroll
+                for (int j = 0; j < kW; ++j) y[j] = tanhf(y[j]);
+                if (A.noise != nullptr && row_valid) {            // actor exploration: y + sigma * eps, kept in [-1, 1]
+#pragma unroll
+                  for (int j = 0; j < kW; ++j)
+                    if (n0 + j < L.N) {
+                      const float t = __fadd_rn(y[j], __fmul_rn(sigma_row, __ldg(A.noise + grow * A.out_dim + n0 + j)));
+                      y[j] = fminf(fmaxf(t, -1.0f), 1.0f);
+                    }
+                }
+              }
+              if (row_valid) {
+#pragma unroll
+                for (int j = 0; j < kW; ++j)
+                  if (n0 + j < L.N) A.out[grow * A.out_dim + n0 + j] = y[j];
+              }
+            };
+            for (int s = 0; s < n_slices; ++s) {
+              if (split) head_slice(PathC<16>{}, s * 32 + sub, s + 1 == n_slices);
+              else head_slice(PathC<32>{}, s * 32, s + 1 == n_slices);
             }
           }
         }
