@@ -34,7 +34,7 @@ INT8_OVER_BF16 = 2.0     # nominal dense tensor ratio (4.5 POPS int8 vs 2.25 PFL
 # bytes read + written at the captured batch, captured batch, bytes that do not scale with the rows
 # (weight images, read from DRAM once per launch).
 NCU_TRAFFIC = {
-    "mlp_wide": ("fused_mlp_pair_kernel (forward)", "mlp_fused_pair.cu", "ec865bb3aaf97e9da53adecae889c597a8b8837a", 22.842624e6, 37888, 3.4e6),
+    "mlp_wide": ("fc_pair_kernel x 5 layers (forward; the observation quantizer's 42 MB not captured)", "fc_pair.cu", "4600641b44279fc762de32b451df04b04a39de68", 393.8e6, 65536, 3.4e6),
     "actorq_2048": ("fc_pair_kernel x layers (forward)", "fc_pair.cu", "2308d1a418591197491457222fe768ff86e5e879", 717e6, 65536, 8.6e6),
 }
 
@@ -516,7 +516,7 @@ def main():
         peak = INT8_OVER_BF16 * float(peaks["bf16_tflops"])
         kernel_name, traffic, traffic_note = ncu_traffic(args.workload, batch)
         if kernel_name is None:
-            wide = max(l.out_features for l in spec.layers[:-1]) > 1024
+            wide = max(l.out_features for l in spec.layers[:-1]) > 512
             kernel_name = ("conv layer kernels (forward)" if spec.obs_dtype != "f32" else
                            "fc_pair_kernel x layers (forward)" if wide else "fused MLP kernel (forward)")
         # denominator: the INT8 tensor rate measured in this process by the library's bare MMA loop
