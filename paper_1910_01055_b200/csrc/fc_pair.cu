@@ -61,6 +61,7 @@ struct Args {
   int K, N, Kpad, Npad, nkb, nchunk, nkb_out;
   int a_unsigned, out_unsigned;
   int last, head;
+  int reverse;             // walk the tile pairs from the last one down: the layer before wrote those last, they are the ones still in L2
   long long batch, n_tile_pairs, n_items;
   float *out;
   int *actions;
@@ -145,7 +146,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
     long long tp = tp_first;
     int c = c_first;
     for (long long item = pair_idx; item < A.n_items && ok; item += n_pairs) {
-      const long long tile = 2 * tp + rank;
+      const long long tile = 2 * (A.reverse ? A.n_tile_pairs - 1 - tp : tp) + rank;
       const int rows_c = min(kAccCols, A.Npad - c * kAccCols);
       const int half_rows = rows_c >> 1;
       const int n_first = c * kAccCols + (int)rank * half_rows;     // weight rows [n_first, + half_rows)
@@ -263,7 +264,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
       t2 = t + tp_step; c2 = cc + c_step;
       if (c2 >= A.nchunk) { c2 -= A.nchunk; ++t2; }
     };
-    auto fetch_rs = [&](long long t) { return __ldg(A.rs_in + (2 * t + rank) * kTileM + row); };
+    auto fetch_rs = [&](long long t) { return __ldg(A.rs_in + (2 * (A.reverse ? A.n_tile_pairs - 1 - t : t) + rank) * kTileM + row); };
     auto fetch_cc = [&](int cc) {     // (the array is zero-padded to a multiple of 128 entries; chunks may end earlier)
       const int n = cc * kAccCols + part * kPartCols + 4 * lane;
       return (n < ((A.N + 127) & ~127)) ? __ldg(reinterpret_cast<const int4 *>(A.cc + n)) : make_int4(0, 0, 0, 0);
@@ -273,7 +274,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
     if (pair_idx < A.n_items) { rs_next = fetch_rs(tp); cc_next = fetch_cc(c); }
     for (long long item = pair_idx; item < A.n_items && ok; item += n_pairs, ++it, tp = tp_nx, c = c_nx) {
       step(tp, c, tp_nx, c_nx);
-      const long long tile = 2 * tp + rank;
+      const long long tile = 2 * (A.reverse ? A.n_tile_pairs - 1 - tp : tp) + rank;
       const long long grow = tile * kTileM + row;
       const bool row_valid = grow < A.batch;
       const int rs_in = rs_next;
@@ -632,6 +633,7 @@ static int fcp_run_layers(actorq_policy *p, FcpLaunch &F, int l_begin, long long
     A.nchunk = (A.Npad + fcp::kAccCols - 1) / fcp::kAccCols;
     A.nkb_out = (L.g.N + 127) / 128;
     A.last = last ? 1 : 0;
+    A.reverse = (l - l_begin) & 1;       // alternate directions: a layer starts where the one before it ended
     A.head = p->head;
     A.batch = batch;
     A.n_tile_pairs = n_tile_pairs;
