@@ -18,8 +18,9 @@
 //     MMAs have finished reading the layer's input before the epilogue starts, so the next layer's
 //     input codes overwrite it in place (one A buffer per slot);
 //   - column constants and per-layer parameters of every layer are loaded into shared memory once;
-//   - the head's fp32 rows leave through shared memory (the slot's dead A buffer) as contiguous
-//     runs, with tanh / exploration noise applied during the copy-out, spread evenly over the threads.
+//   - the head: a thread applies Eq. 3, tanh and the exploration noise to 8 columns of its row at a
+//     time (8 independent chains) and stores them itself (the outputs are a few KB per tile: staging
+//     them in shared memory for coalesced stores cost two rendezvous per tile and was slower).
 // Roles per CTA (704 threads): warp 0 bulk-copy producer, warp 1 MMA issuer (even CTA) / relay of
 // "my half of the weights has landed" (odd CTA), warps 2-5 observation quantizers, warps 6-21
 // epilogue (four per tensor-memory lane quarter, each a quarter of a layer's columns: the requantizer
@@ -72,7 +73,6 @@ struct Args {
   int head;
   float obs_inv_s;         // input quantizer of the observations (host-known: 1 / s_a and z_a of layer 0)
   int obs_z;
-  uint32_t head_magic;     // ceil(2^32 / out_dim): floor(i / out_dim) = umulhi(i, head_magic) for the small i of the copy-out
   int obs_dim, out_dim;
   int w_bytes;             // resident weights per CTA
   int a_bytes;             // one hidden-activation buffer (per slot)
@@ -90,7 +90,6 @@ struct __align__(16) Barriers {
   uint64_t stage_full, stage_empty;
   uint64_t a0_full[2], a0_empty[2];
   uint64_t acc_full[2], a_ready[2];
-  uint64_t qbar[4];          // the epilogue warps of a lane quarter meet here around the head's copy-out
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
@@ -183,7 +182,6 @@ fused_mlp_resident_kernel(const __grid_constant__ Args A) {
       mbar_init(&bars->acc_full[s], 1);
       mbar_init(&bars->a_ready[s], 2 * kEpiWarps);
     }
-    for (int q = 0; q < 4; ++q) mbar_init(&bars->qbar[q], kParts);
     mbar_init(&bars->drain, 1);
     bars->abort_flag = 0;
     if (blockIdx.x == 0) A.status[7] = (int)smem_u32(bars);
@@ -376,16 +374,8 @@ fused_mlp_resident_kernel(const __grid_constant__ Args A) {
       for (int i = et; i < Lc.Npad; i += kEpiWarps * 32) cc_smem[Lc.cc_off + i] = (i < Lc.N) ? __ldg(Lc.cc + i) : 0;
     }
     named_bar_sync(1, kEpiWarps * 32);
-    uint32_t af_cnt[2] = {0, 0}, q_cnt = 0;
+    uint32_t af_cnt[2] = {0, 0};
     bool ok = true;
-    // the four warps of a lane quarter meet (bounded, like every other wait)
-    auto quarter_sync = [&]() -> bool {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->qbar[quarter]);
-      const bool met = __all_sync(0xffffffffu, mbar_wait(&bars->qbar[quarter], q_cnt & 1, abort_flag, A.status));
-      ++q_cnt;
-      return met;
-    };
     for (int j0 = 0; j0 < T && ok; j0 += 2) {
       const int ns = min(2, T - j0);
       for (int l = 0; l < A.n_layers && ok; ++l) {
@@ -481,21 +471,19 @@ fused_mlp_resident_kernel(const __grid_constant__ Args A) {
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(a_ready_leader + 8u * (uint32_t)s);
           } else {
-            // ---- head: Eq. 3 on the accumulator; the rows leave through the slot's A buffer ----
-            // Each quarter stages its 32 rows in the bytes its own rows occupy in that buffer (4 KB per
-            // K block), rows Ns = N | 1 floats apart (odd: conflict-free stores), then its two warps
-            // copy them out as one contiguous run, applying tanh / exploration noise on the way.
-            const int N = L.N, Ns = N | 1;
-            auto stage_at = [&](int i) -> float * {      // staged element i = staged row * Ns + column
-              return reinterpret_cast<float *>(a_out + ((uint32_t)(i >> 10) << 14) + quarter * 4096 + ((i & 1023) << 2));
-            };
+            // ---- head: Eq. 3 on the accumulator, tanh, exploration noise, stores ----
+            const int N = L.N;
             // warp `part` of the quarter dequantizes 8 columns of every 32; a greedy-action head is done by
             // one warp per quarter, which sees whole rows (lowest index among equal maxima)
             const bool greedy = A.head == ACTORQ_HEAD_ARGMAX;
             if (!greedy || part == 0) {
               float best_v = 0.0f;
               int best_n = -1;
-              for (int n0 = greedy ? 0 : part * 8; n0 < N; n0 += greedy ? 8 : 32) {
+              const bool noisy = A.head == ACTORQ_HEAD_TANH && (A.noise != nullptr || A.noise_seeded);
+              const float sigma_row = (noisy && row_valid) ? __ldg(A.sigma + grow) : 0.0f;
+              // (n0 = 8 nb: the two Philox blocks of a thread's 8 columns are then visibly 2 nb and 2 nb + 1)
+              for (int nb = greedy ? 0 : part; nb * 8 < N; nb += greedy ? 1 : kParts) {
+                const int n0 = nb * 8;
                 uint32_t r[8];
                 tmem_ld8_wait(acc_addr + n0, r);
                 const int4 c0 = *reinterpret_cast<const int4 *>(cc_smem + L.cc_off + n0);
@@ -509,50 +497,30 @@ fused_mlp_resident_kernel(const __grid_constant__ Args A) {
                   y[j] = __fmul_rn(__int2float_rn(acc), p.P);                     // Eq. 3
                   if (greedy && n0 + j < N && (y[j] > best_v || best_n < 0)) { best_v = y[j]; best_n = n0 + j; }
                 }
+                if (A.head == ACTORQ_HEAD_TANH) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                  if (n0 + j < N) *stage_at(lane * Ns + n0 + j) = y[j];
+                  for (int j = 0; j < 8; ++j) y[j] = tanhf(y[j]);
+                  if (noisy && row_valid) {                           // actor exploration: y + sigma * eps, kept in [-1, 1]
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                      if (n0 + j < N) {
+                        const float e = A.noise_seeded ? exploration_normal(A.seed_lo, A.seed_hi, A.noise_row0 + grow, nb * 8 + j)
+                                                       : __ldg(A.noise + grow * N + n0 + j);
+                        y[j] = fminf(fmaxf(__fadd_rn(y[j], __fmul_rn(sigma_row, e)), -1.0f), 1.0f);
+                      }
+                  }
+                }
+                if (row_valid) {
+#pragma unroll
+                  for (int j = 0; j < 8; ++j)
+                    if (n0 + j < N) A.out[grow * N + n0 + j] = y[j];
+                }
               }
               if (greedy && row_valid) A.actions[grow] = best_n;
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(a_ready_leader + 8u * (uint32_t)s);    // the accumulator is free
-            ok = quarter_sync();
-            if (!ok) break;
-            const long long q_row0 = tile_row0 + quarter * 32;
-            const int valid_q = (int)max(0ll, min(32ll, A.batch - q_row0));
-            const int total = valid_q * N;
-            float *dst = A.out + q_row0 * N;
-            const int t128 = part * 32 + lane;
-            // element i of the quarter's run = staged row i / N, column i % N (the division by a multiply
-            // with ceil(2^32 / N), exact for these small i); two elements per thread in flight
-            for (int i0 = t128; i0 < total; i0 += 2 * 32 * kParts) {
-              const int i1 = i0 + 32 * kParts;
-              const int r0 = (int)__umulhi((uint32_t)i0, A.head_magic), r1 = (int)__umulhi((uint32_t)i1, A.head_magic);
-              float y0 = *stage_at(r0 * Ns + (i0 - r0 * N));
-              float y1 = (i1 < total) ? *stage_at(r1 * Ns + (i1 - r1 * N)) : 0.0f;
-              if (A.head == ACTORQ_HEAD_TANH) {
-                y0 = tanhf(y0);
-                y1 = tanhf(y1);
-                if (A.noise != nullptr || A.noise_seeded) {          // actor exploration: y + sigma * eps, kept in [-1, 1]
-                  const float e0 = A.noise_seeded ? exploration_normal(A.seed_lo, A.seed_hi, A.noise_row0 + q_row0 + r0, i0 - r0 * N)
-                                                  : __ldg(A.noise + q_row0 * N + i0);
-                  y0 = __fadd_rn(y0, __fmul_rn(__ldg(A.sigma + q_row0 + r0), e0));
-                  y0 = fminf(fmaxf(y0, -1.0f), 1.0f);
-                  if (i1 < total) {
-                    const float e1 = A.noise_seeded ? exploration_normal(A.seed_lo, A.seed_hi, A.noise_row0 + q_row0 + r1, i1 - r1 * N)
-                                                    : __ldg(A.noise + q_row0 * N + i1);
-                    y1 = __fadd_rn(y1, __fmul_rn(__ldg(A.sigma + q_row0 + r1), e1));
-                    y1 = fminf(fmaxf(y1, -1.0f), 1.0f);
-                  }
-                }
-              }
-              dst[i0] = y0;
-              if (i1 < total) dst[i1] = y1;
-            }
-            ok = quarter_sync();                  // the staged rows are read before the slot's next codes overwrite them
-            if (!ok) break;
           }
         }
       }
@@ -591,8 +559,6 @@ static ResPlan plan_resident(const actorq_policy *p) {
     pl.w_bytes += nkb * (res_round_up(g.N, 32) / 2) * 128;
     pl.cc_ints += res_round_up(g.N, 32);
   }
-  const int n_head = p->layers[p->n_layers - 1].g.N;
-  if (32 * (n_head | 1) * 4 > 4096 * a_blocks) return pl;       // the head's rows are staged in a slot's A buffer
   pl.a_bytes = a_blocks * kStageBytes;
   pl.a0_bytes = ((p->layers[0].g.K + 127) / 128) * kStageBytes;
   const int misc = (int)sizeof(res::Barriers) + (8 + 16) * kTileM * (int)sizeof(int16_t) +
@@ -687,7 +653,6 @@ int launch_forward_fused_resident(actorq_policy *p, const void *obs, long long b
   A.out_dim = p->layers[p->n_layers - 1].g.N;
   A.obs_inv_s = p->act[0].inv_s;
   A.obs_z = p->act[0].z;
-  A.head_magic = (uint32_t)((0x100000000ull + (unsigned long long)A.out_dim - 1) / (unsigned long long)A.out_dim);
   A.w_bytes = pl.w_bytes;
   A.a_bytes = pl.a_bytes;
   A.a0_bytes = pl.a0_bytes;
