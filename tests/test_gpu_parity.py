@@ -478,6 +478,34 @@ def test_wide_fc_policies_run_on_the_layer_kernel(dims, head):
     pol.close()
 
 
+@pytest.mark.parametrize("dims,head,Bsz", [([128, 1024, 1024, 1024, 32], "tanh", 1300),     # 6 tile pairs, the last one half empty
+                                           ([40, 640, 520, 7], "argmax", 3),                # a handful of rows, greedy head
+                                           ([33, 1024, 96, 12], "linear", 769)])            # 4 tile pairs, the odd tile of the last one missing
+def test_policies_wider_than_512_default_to_the_layer_kernel(dims, head, Bsz):
+    """A policy the fused kernels could take but with a hidden layer wider than 512 runs on the layer
+    kernel unless a fused kernel is pinned: launch count = input quantizer + one launch per layer; every
+    layer's accumulators and codes and the outputs against the checker (successive layers walk the
+    tile pairs in opposite directions: odd and even tile-pair counts, ragged last tiles); and the pinned
+    fused kernel gives the same outputs bit for bit."""
+    spec = W.calibrate(W.mlp_policy("w", dims, seed=91, head=head, nonzero_bias=True), 64, seed=91)
+    pol, qp, _ = _quantize_both(spec)
+    obs = W.make_obs(spec, Bsz, seed=91)
+    out, act = pol.forward(torch.from_numpy(obs).cuda())
+    torch.cuda.synchronize()
+    assert pol.status() == B.OK
+    assert B.actorq_policy_last_launch_count(pol.handle) == len(dims)
+    _check_forward(pol, qp, spec, obs)
+    B.actorq_policy_set_fused_variant(pol.handle, 2)
+    other, other_act = pol.forward(torch.from_numpy(obs).cuda())
+    torch.cuda.synchronize()
+    assert pol.status() == B.OK
+    assert B.actorq_policy_last_launch_count(pol.handle) == 1
+    assert torch.equal(out, other)
+    if head == "argmax":
+        assert torch.equal(act, other_act)
+    pol.close()
+
+
 @pytest.mark.parametrize("dims,head,Bsz", [([24, 256, 256, 256, 6], "tanh", 200),
                                            ([50, 416, 300, 160, 9], "linear", 700),      # chunk halves that straddle weight tiles
                                            ([33, 96, 520, 1000, 40, 3], "tanh", 385),    # narrow, ragged and 5 layers
