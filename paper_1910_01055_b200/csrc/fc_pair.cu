@@ -59,6 +59,8 @@ struct Args {
   const LayerParams *params;
   int layer;
   int K, N, Kpad, Npad, nkb, nchunk, nkb_out;
+  int chunk_cols;          // output columns per work item: 256, or 128 / 64 when a layer has fewer items than CTA pairs
+
   int a_unsigned, out_unsigned;
   int last, head;
   int reverse;             // walk the tile pairs from the last one down: the layer before wrote those last, they are the ones still in L2
@@ -147,9 +149,9 @@ fc_pair_kernel(const __grid_constant__ Args A) {
     int c = c_first;
     for (long long item = pair_idx; item < A.n_items && ok; item += n_pairs) {
       const long long tile = 2 * (A.reverse ? A.n_tile_pairs - 1 - tp : tp) + rank;
-      const int rows_c = min(kAccCols, A.Npad - c * kAccCols);
+      const int rows_c = min(A.chunk_cols, A.Npad - c * A.chunk_cols);
       const int half_rows = rows_c >> 1;
-      const int n_first = c * kAccCols + (int)rank * half_rows;     // weight rows [n_first, + half_rows)
+      const int n_first = c * A.chunk_cols + (int)rank * half_rows;     // weight rows [n_first, + half_rows)
       const int t0 = n_first >> 7, r0 = n_first & 127;
       const int rows_a = min(half_rows, 128 - r0);                  // rows taken from image tile t0
       const int rows_b = half_rows - rows_a;                        // the rest, from the next tile
@@ -184,7 +186,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
     bool ok = true;
     int c = c_first;
     for (long long item = pair_idx; item < A.n_items && ok; item += n_pairs, ++it) {
-      const int rows_c = min(kAccCols, A.Npad - c * kAccCols);
+      const int rows_c = min(A.chunk_cols, A.Npad - c * A.chunk_cols);
       c += c_step;
       if (c >= A.nchunk) c -= A.nchunk;
       const uint32_t idesc = instr_desc_pair(rows_c, A.a_unsigned != 0);
@@ -266,7 +268,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
     };
     auto fetch_rs = [&](long long t) { return __ldg(A.rs_in + (2 * (A.reverse ? A.n_tile_pairs - 1 - t : t) + rank) * kTileM + row); };
     auto fetch_cc = [&](int cc) {     // (the array is zero-padded to a multiple of 128 entries; chunks may end earlier)
-      const int n = cc * kAccCols + part * kPartCols + 4 * lane;
+      const int n = cc * A.chunk_cols + part * kPartCols + 4 * lane;
       return (n < ((A.N + 127) & ~127)) ? __ldg(reinterpret_cast<const int4 *>(A.cc + n)) : make_int4(0, 0, 0, 0);
     };
     int rs_next = 0;
@@ -282,7 +284,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
       cc_warp[lane] = cc_next;
       __syncwarp();
       if (item + n_pairs < A.n_items) { rs_next = fetch_rs(tp_nx); cc_next = fetch_cc(c_nx); }
-      const int rows_c = min(kAccCols, A.Npad - c * kAccCols);
+      const int rows_c = min(A.chunk_cols, A.Npad - c * A.chunk_cols);
       const uint32_t buf = it & 1, use = it >> 1;
       const uint32_t acc = tmem + lane_addr + buf * kAccCols;
       const int rterm = -p.z_w * rs_in;
@@ -320,7 +322,7 @@ fc_pair_kernel(const __grid_constant__ Args A) {
             }
           }
           const uint32_t (&r)[32] = rr[s & 1];
-          const int n0 = c * kAccCols + col0;
+          const int n0 = c * A.chunk_cols + col0;
           const int4 *cc4 = cc_warp + s * 8;
           uint32_t packed[8];
           if (kPath == 0) requant32_u8<false>(r, cc4, (uint32_t)rterm + 0x4B000000u, Ms, cs, packed);
@@ -630,7 +632,11 @@ static int fcp_run_layers(actorq_policy *p, FcpLaunch &F, int l_begin, long long
     A.Kpad = fcp_round_up(L.g.K, 32);
     A.Npad = fcp_round_up(L.g.N, 32);
     A.nkb = (L.g.K + 127) / 128;
-    A.nchunk = (A.Npad + fcp::kAccCols - 1) / fcp::kAccCols;
+    // a layer with fewer (tile pair, 256 columns) items than CTA pairs is cut into narrower items: more
+    // pairs work, and an item's K loop is shorter per MMA (a K loop cannot be shorter than its MMA count)
+    A.chunk_cols = fcp::kAccCols;
+    while (A.chunk_cols > 64 && !last && n_tile_pairs * ((A.Npad + A.chunk_cols - 1) / A.chunk_cols) < F.max_pairs) A.chunk_cols >>= 1;
+    A.nchunk = (A.Npad + A.chunk_cols - 1) / A.chunk_cols;
     A.nkb_out = (L.g.N + 127) / 128;
     A.last = last ? 1 : 0;
     A.reverse = (l - l_begin) & 1;       // alternate directions: a layer starts where the one before it ended
