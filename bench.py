@@ -34,8 +34,8 @@ INT8_OVER_BF16 = 2.0     # nominal dense tensor ratio (4.5 POPS int8 vs 2.25 PFL
 # bytes read + written at the captured batch, captured batch, bytes that do not scale with the rows
 # (weight images, read from DRAM once per launch).
 NCU_TRAFFIC = {
-    "mlp_wide": ("fc_pair_kernel x 5 layers (forward; the observation quantizer's 42 MB not captured)", "fc_pair.cu", "95295712d71d328e2b58c66d7a54df2b05eca3b3", 395.8e6, 65536, 3.4e6),
-    "actorq_2048": ("fc_pair_kernel x 4 layers (forward; the observation quantizer not captured)", "fc_pair.cu", "95295712d71d328e2b58c66d7a54df2b05eca3b3", 711.8e6, 65536, 8.6e6),
+    "mlp_wide": ("fc_pair_kernel x 5 layers (forward; the observation quantizer's 42 MB not captured)", "fc_pair.cu", "fd7f06d8a8ee647fdf92e523331e55c23ba52ea9", 394.2e6, 65536, 3.4e6),
+    "actorq_2048": ("fc_pair_kernel x 4 layers (forward; the observation quantizer not captured)", "fc_pair.cu", "fd7f06d8a8ee647fdf92e523331e55c23ba52ea9", 718.7e6, 65536, 8.6e6),
 }
 
 
